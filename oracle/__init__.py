@@ -1,0 +1,164 @@
+"""CPU oracle: test infrastructure only.
+
+numpy-facing wrappers around ``oracle.c`` (see its header for what each
+function follows in the paper).  Nothing here imports or calls the CUDA
+library, and no product code may import this package: only tests, the smoke
+check and the benchmark's CPU-baseline leg do.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from dataclasses import dataclass
+
+import numpy as np
+
+from .build import build as _build
+
+DENSE, COMPRESSED = 0, 1
+_MAXR = 8
+_P64 = C.POINTER(C.c_int64)
+_PD = C.POINTER(C.c_double)
+
+
+class _Storage(C.Structure):
+    _fields_ = [("rank", C.c_int), ("npos", C.c_int64 * _MAXR), ("ncrd", C.c_int64 * _MAXR),
+                ("pos", _P64 * _MAXR), ("crd", _P64 * _MAXR), ("nval", C.c_int64), ("val", _PD),
+                ("entry_pos", _P64)]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(_build())
+        _lib.orc_unpack.restype = C.c_int64
+    return _lib
+
+
+def _i64(a):
+    return np.ascontiguousarray(a, dtype=np.int64)
+
+
+def _f64(a):
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _ptr(a, t=_P64):
+    return a.ctypes.data_as(t)
+
+
+@dataclass
+class Storage:
+    """pos[l] / crd[l] are int64 arrays (None at dense levels); val is f64."""
+    dims: tuple
+    lt: tuple
+    ord: tuple
+    pos: list
+    crd: list
+    val: np.ndarray
+    entry_pos: np.ndarray
+
+
+def pack(dims, coords, vals, lt, ord=None) -> Storage:
+    """Section 4.1 storage from a coordinate list (coords[d] per logical dim)."""
+    rank = len(dims)
+    ord = tuple(range(rank)) if ord is None else tuple(int(o) for o in ord)
+    cs = [_i64(c) for c in coords]
+    v = _f64(vals)
+    nnz = v.size
+    carr = (_P64 * rank)(*[_ptr(c) for c in cs])
+    st = _Storage()
+    rc = lib().orc_pack(C.c_int(rank), _ptr(_i64(dims)), C.c_int64(nnz), carr, _ptr(v, _PD),
+                        (C.c_int * rank)(*[int(t) for t in lt]), (C.c_int * rank)(*ord), C.byref(st))
+    if rc != 0:
+        lib().orc_free_storage(C.byref(st))
+        raise ValueError({-1: "invalid argument", -2: "coordinate out of range", -3: "out of memory"}.get(rc, rc))
+    pos, crd = [], []
+    for l in range(rank):
+        if lt[l] == COMPRESSED:
+            pos.append(np.ctypeslib.as_array(st.pos[l], (st.npos[l],)).copy())
+            crd.append(np.ctypeslib.as_array(st.crd[l], (st.ncrd[l],)).copy() if st.ncrd[l] else np.empty(0, np.int64))
+        else:
+            pos.append(None)
+            crd.append(None)
+    val = np.ctypeslib.as_array(st.val, (st.nval,)).copy() if st.nval else np.empty(0, np.float64)
+    ep = np.ctypeslib.as_array(st.entry_pos, (nnz,)).copy() if nnz else np.empty(0, np.int64)
+    lib().orc_free_storage(C.byref(st))
+    return Storage(tuple(int(d) for d in dims), tuple(int(t) for t in lt), ord, pos, crd, val, ep)
+
+
+def unpack(s: Storage):
+    """Stored entries in storage order as (logical coords per dim, values)."""
+    rank = len(s.dims)
+    st = _Storage()
+    st.rank = rank
+    keep = []
+    for l in range(rank):
+        if s.lt[l] == COMPRESSED:
+            p, c = _i64(s.pos[l]), _i64(s.crd[l])
+            keep += [p, c]
+            st.pos[l], st.crd[l] = _ptr(p), _ptr(c)
+            st.npos[l], st.ncrd[l] = p.size, c.size
+    v = _f64(s.val)
+    st.val, st.nval = _ptr(v, _PD), v.size
+    outs = [np.empty(v.size, np.int64) for _ in range(rank)]
+    vo = np.empty(v.size, np.float64)
+    n = lib().orc_unpack(C.byref(st), _ptr(_i64(s.dims)), (C.c_int * rank)(*s.lt), (C.c_int * rank)(*s.ord),
+                         (_P64 * rank)(*[_ptr(o) for o in outs]), _ptr(vo, _PD))
+    assert n == v.size
+    return outs, vo
+
+
+def _slots(rows, m):
+    if rows is None:
+        return None, m
+    rows = _i64(rows)
+    slot = np.full(m, -1, np.int64)
+    slot[rows] = np.arange(rows.size)
+    return slot, rows.size
+
+
+def spmm(m, ai, ak, av, B, rows=None):
+    """C = A * B over the coordinate list; returns (C, bound) for all rows or the listed ones."""
+    B = _f64(B)
+    N = B.shape[1]
+    slot, ns = _slots(rows, m)
+    Cm = np.empty((ns, N)); bd = np.empty((ns, N))
+    ai, ak, av = _i64(ai), _i64(ak), _f64(av)
+    rc = lib().orc_spmm(C.c_int64(av.size), _ptr(ai), _ptr(ak), _ptr(av, _PD), _ptr(B, _PD), C.c_int64(N),
+                        C.c_int64(N), _ptr(slot) if slot is not None else None, C.c_int64(ns),
+                        _ptr(Cm, _PD), _ptr(bd, _PD))
+    assert rc == 0
+    return Cm, bd
+
+
+def spmv(m, ai, ak, av, x, rows=None):
+    y, b = spmm(m, ai, ak, av, _f64(x).reshape(-1, 1), rows)
+    return y[:, 0], b[:, 0]
+
+
+def sddmm(si, sj, sv, A, B):
+    """x_e = S_e * sum_k A[i_e,k] B[k,j_e], one value per listed entry (input order)."""
+    A, B = _f64(A), _f64(B)
+    si, sj, sv = _i64(si), _i64(sj), _f64(sv)
+    x = np.empty(sv.size); bd = np.empty(sv.size)
+    rc = lib().orc_sddmm(C.c_int64(sv.size), _ptr(si), _ptr(sj), _ptr(sv, _PD), _ptr(A, _PD), C.c_int64(A.shape[1]),
+                         _ptr(B, _PD), C.c_int64(B.shape[1]), C.c_int64(A.shape[1]), _ptr(x, _PD), _ptr(bd, _PD))
+    assert rc == 0
+    return x, bd
+
+
+def mttkrp(I, ti, tj, tk, tv, B, Cf, rows=None):
+    """M[i,r] = sum T[i,j,k] B[j,r] C[k,r]; returns (M, bound)."""
+    B, Cf = _f64(B), _f64(Cf)
+    R = B.shape[1]
+    slot, ns = _slots(rows, I)
+    M = np.empty((ns, R)); bd = np.empty((ns, R))
+    ti, tj, tk, tv = _i64(ti), _i64(tj), _i64(tk), _f64(tv)
+    rc = lib().orc_mttkrp(C.c_int64(tv.size), _ptr(ti), _ptr(tj), _ptr(tk), _ptr(tv, _PD), _ptr(B, _PD),
+                          _ptr(Cf, _PD), C.c_int64(R), _ptr(slot) if slot is not None else None, C.c_int64(ns),
+                          _ptr(M, _PD), _ptr(bd, _PD))
+    assert rc == 0
+    return M, bd

@@ -1,0 +1,18 @@
+"""Compile the CPU oracle (plain C) into oracle/liboracle.so.  Test infrastructure only."""
+import os
+import subprocess
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+SRC = os.path.join(HERE, "oracle.c")
+LIB = os.path.join(HERE, "liboracle.so")
+
+
+def build(force: bool = False) -> str:
+    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= os.path.getmtime(SRC):
+        return LIB
+    subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-fPIC", "-shared", "-o", LIB, SRC, "-lm"])
+    return LIB
+
+
+if __name__ == "__main__":
+    print(build(force=True))
