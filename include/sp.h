@@ -1,0 +1,173 @@
+/*
+ * sp.h - C ABI of the sparse tensor library (CUDA, sm_100a, one GPU).
+ *
+ * The calls follow the statement of the problem in "Compiler Support for Sparse
+ * Tensor Computations in MLIR" (arXiv 2202.04305): a tensor is stored according
+ * to an encoding (Section 4.1: per-level type dense | compressed, a dimension
+ * ordering, and bit widths for pointers and indices) as the arrays
+ * pointers[l][*], indices[l][*] and values[*]; storage is built from a
+ * coordinate list (Section 4.2: conversions go through an intermediate
+ * coordinate scheme); and the kernels are the tensor index expressions the
+ * paper runs over that storage (Sections 1, 6.2, 6.3).
+ *
+ * Naming: "positions" = the paper's pointers, "coordinates" = its indices.
+ * A "level" l is a storage level; dimOrdering[l] is the logical dimension kept
+ * at level l.
+ *
+ * Conventions for every call
+ *   - All data pointers are DEVICE pointers owned by the caller unless the
+ *     parameter says "host".  The library owns only what lives inside an
+ *     sp_tensor (released by sp_free) and transient workspaces that it obtains
+ *     and returns through the allocator (sp_set_allocator).
+ *   - Dense operands are row-major f64 with a leading dimension in elements.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Kernel calls are asynchronous on it.  sp_pack synchronises the stream
+ *     (the sizes of the level arrays depend on the data).
+ *   - Kernels OVERWRITE their output.
+ *   - Every call returns an sp_status; nothing throws across the boundary.
+ *     An encoding a kernel does not handle yields SP_ERR_UNSUPPORTED, never a
+ *     different algorithm on the host.
+ *   - A handle is immutable after sp_pack.  Kernels cache work-partition tables
+ *     inside it on first use; use a handle from one stream at a time.
+ */
+#ifndef SP_H
+#define SP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SP_MAX_RANK 3
+
+typedef struct sp_tensor sp_tensor;   /* opaque; owns device arrays */
+
+typedef enum { SP_DENSE = 0, SP_COMPRESSED = 1 } sp_level_type;
+
+typedef enum {
+    SP_OK = 0,
+    SP_ERR_INVALID_ARG = 1,     /* null pointer, bad rank, dimOrdering not a permutation, bad width */
+    SP_ERR_UNSUPPORTED = 2,     /* encoding / shape not handled by this call */
+    SP_ERR_OUT_OF_RANGE = 3,    /* a coordinate is < 0 or >= its dimension */
+    SP_ERR_WIDTH_OVERFLOW = 4,  /* a position or coordinate does not fit the requested width */
+    SP_ERR_DUPLICATE = 5,       /* SP_DUP_ERROR was set and two entries share coordinates */
+    SP_ERR_ALLOC = 6,           /* the allocator returned NULL */
+    SP_ERR_CUDA = 7,            /* a CUDA runtime call failed */
+    SP_ERR_TIMEOUT = 8          /* a bounded device-side wait ran out */
+} sp_status;
+
+/* flags of sp_pack */
+#define SP_DUP_SUM   0u   /* entries with equal coordinates are added, in input order (default) */
+#define SP_DUP_ERROR 1u   /* ... are reported as SP_ERR_DUPLICATE instead */
+
+const char* sp_status_string(sp_status s);
+
+/*
+ * Workspace and storage allocator.  alloc(bytes, stream, ctx) returns device
+ * memory usable on `stream`; dealloc returns it.  Both NULL restores the
+ * default (cudaMalloc / cudaFree).  Process-wide; set it before the first
+ * sp_pack and do not change it while handles are alive.
+ */
+sp_status sp_set_allocator(void* (*alloc)(size_t bytes, void* stream, void* ctx),
+                           void (*dealloc)(void* ptr, void* stream, void* ctx), void* ctx);
+
+/*
+ * sp_pack - build the storage of Section 4.1 from an unsorted coordinate list
+ * (Section 4.2: the sparse constant given as index tuples plus values, and
+ * conversion through a coordinate scheme).
+ *
+ *   rank            1..SP_MAX_RANK
+ *   dims            host, rank logical extents (each >= 1)
+ *   nnz             number of entries (>= 0, < 2^32)
+ *   coo_coords      host array of `rank` DEVICE pointers; coo_coords[d][e] is
+ *                   entry e's coordinate in logical dimension d
+ *   coo_coord_bits  32 (int32) or 64 (int64) element type of those arrays
+ *   coo_vals        device, nnz doubles
+ *   dimLevelType    host, per level
+ *   dimOrdering     host, per level: logical dimension stored at level l; NULL = identity
+ *   posBits/crdBits 0 (= 64, the "native" width), 32 or 64; stored unsigned
+ *   flags           SP_DUP_SUM or SP_DUP_ERROR
+ *   out             receives the handle; release with sp_free
+ *
+ * Stored entries appear in lexicographic order of their level coordinates;
+ * empty parents repeat their position; trailing dense levels materialise
+ * explicit zeros (the paper's five storage examples).  Explicit zeros in the
+ * input are kept.  The inputs are not modified.
+ */
+sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz,
+                  const void* const* coo_coords, int coo_coord_bits, const double* coo_vals,
+                  const sp_level_type* dimLevelType, const int* dimOrdering,
+                  int posBits, int crdBits, unsigned flags, void* stream, sp_tensor** out);
+
+/* Releases the handle and its device arrays (NULL is allowed). */
+sp_status sp_free(sp_tensor* t);
+
+/*
+ * Accessors - the paper's pointers / indices / values operations (Section 4.2),
+ * each returning one level's array as a device pointer plus its length in
+ * elements.  Dense levels have no arrays: *dev_ptr = NULL, *len = 0.
+ * Element type is uint32_t or uint64_t according to the handle's widths.
+ * Any output pointer of sp_info may be NULL.
+ */
+sp_status sp_info(const sp_tensor* t, int* rank, int64_t* dims /* host, rank */,
+                  sp_level_type* dimLevelType, int* dimOrdering, int* posBits, int* crdBits);
+sp_status sp_positions(const sp_tensor* t, int level, const void** dev_ptr, int64_t* len);
+sp_status sp_coordinates(const sp_tensor* t, int level, const void** dev_ptr, int64_t* len);
+sp_status sp_values(const sp_tensor* t, const double** dev_ptr, int64_t* len);
+
+/*
+ * sp_unpack - storage back to a coordinate list (the other half of
+ * Section 4.2's conversion through coordinates).  Emits every stored value in
+ * storage order with its LOGICAL coordinates, explicit zeros included.
+ * coo_coords_out: host array of `rank` device pointers to int64 arrays with
+ * room for sp_values' len entries each; vals_out likewise.  *nnz_out (host)
+ * receives the count.
+ */
+sp_status sp_unpack(const sp_tensor* t, void* const* coo_coords_out, double* vals_out,
+                    int64_t* nnz_out, void* stream);
+
+/*
+ * sp_spmv - y[i] = sum_k A[i,k] * x[k]  (the matvec of Section 6.2).
+ * A: rank 2, level types (dense, compressed) or (compressed, compressed),
+ * either ordering (CSR, DCSR, CSC, DCSC).  x has dims[1] entries, y dims[0].
+ * Rows without stored entries are written as 0.  Column-major encodings
+ * accumulate with floating-point atomics: the summation order, and so the
+ * last bits, may differ from run to run.
+ */
+sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* stream);
+
+/*
+ * sp_spmm - C[i,j] = sum_k A[i,k] * B[k,j], A sparse, B and C dense
+ * (Sections 1 and 5.2).  B is dims[1] x N with leading dimension ldb, C is
+ * dims[0] x N with ldc.  Encodings and the atomics remark as for sp_spmv.
+ */
+sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t ldb,
+                  double* C, int64_t ldc, void* stream);
+
+/*
+ * sp_sddmm - X[i,j] = S[i,j] * sum_k A[i,k] * B[k,j] for the stored (i,j) of
+ * S (Section 6.2).  S: rank 2, (dense|compressed, compressed), identity
+ * ordering.  A is dims[0] x K (lda), B is K x dims[1] (ldb).  x_vals receives
+ * one value per stored entry of S, in S's storage order (X shares S's
+ * positions and coordinates); its length is sp_values' len.
+ */
+sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const double* B, int64_t ldb,
+                   int64_t K, double* x_vals, void* stream);
+
+/*
+ * sp_mttkrp - M[i,r] = sum_{j,k} T[i,j,k] * B[j,r] * C[k,r]  (Section 6.3,
+ * where the same expression is written A[i,j] = B[i,k,l] * D[l,j] * C[k,j]).
+ * T: rank 3, level types (compressed|dense, compressed, compressed) with
+ * logical dimension 0 at level 0 and the other two in either order.
+ * B is dims[1] x R, C is dims[2] x R, M is dims[0] x R, all contiguous
+ * row-major.  Slices without stored entries give zero rows.
+ */
+sp_status sp_mttkrp(sp_tensor* T, const double* B, const double* C, int64_t R,
+                    double* M, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SP_H */

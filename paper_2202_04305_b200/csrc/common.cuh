@@ -1,0 +1,117 @@
+// Shared host/device declarations of the sparse tensor library (internal).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <map>
+#include <mutex>
+#include <vector>
+
+#include "sp.h"
+
+// ---------------------------------------------------------------------------
+// Handle
+// ---------------------------------------------------------------------------
+
+// Work-partition table cached in a handle: chunk w covers merge-path
+// coordinates [(row[w], nz[w]), (row[w+1], nz[w+1])).
+struct sp_partition {
+    int64_t nchunks = 0;
+    int64_t* row = nullptr;   // nchunks + 1 entries (device)
+    int64_t* nz = nullptr;    // nchunks + 1 entries (device)
+    int64_t* aux = nullptr;   // kernel-specific (MTTKRP: slice of each chunk start)
+    double* carry = nullptr;  // kernel-specific scratch sized by the creator
+    int64_t carry_elems = 0;
+};
+
+struct sp_tensor {
+    int rank = 0;
+    int64_t dims[SP_MAX_RANK] = {0, 0, 0};
+    int lt[SP_MAX_RANK] = {0, 0, 0};
+    int ord[SP_MAX_RANK] = {0, 1, 2};
+    int posBits = 64, crdBits = 64;
+    void* pos[SP_MAX_RANK] = {nullptr, nullptr, nullptr};
+    int64_t npos[SP_MAX_RANK] = {0, 0, 0};
+    void* crd[SP_MAX_RANK] = {nullptr, nullptr, nullptr};
+    int64_t ncrd[SP_MAX_RANK] = {0, 0, 0};
+    double* val = nullptr;
+    int64_t nval = 0;
+    int device = 0;
+    std::mutex mu;
+    std::map<uint64_t, sp_partition> parts;   // key = (kind << 32) | items per chunk
+};
+
+// ---------------------------------------------------------------------------
+// Allocation through the installed allocator
+// ---------------------------------------------------------------------------
+void* sp_dev_alloc(size_t bytes, cudaStream_t stream);
+void sp_dev_free(void* p, cudaStream_t stream);
+
+// Frees everything it handed out when it goes out of scope.
+struct sp_workspace {
+    cudaStream_t stream;
+    std::vector<void*> ptrs;
+    bool failed = false;
+    explicit sp_workspace(cudaStream_t s) : stream(s) {}
+    ~sp_workspace() {
+        for (void* p : ptrs) sp_dev_free(p, stream);
+    }
+    template <typename T>
+    T* get(size_t count) {
+        void* p = sp_dev_alloc((count ? count : 1) * sizeof(T), stream);
+        if (!p) { failed = true; return nullptr; }
+        ptrs.push_back(p);
+        return static_cast<T*>(p);
+    }
+    // Hands ownership of p to the caller (it will not be freed here).
+    void release(void* p) {
+        for (auto& q : ptrs) if (q == p) { q = nullptr; }
+    }
+};
+
+#define SP_CUDA(call)                                   \
+    do {                                                \
+        cudaError_t e__ = (call);                       \
+        if (e__ != cudaSuccess) return SP_ERR_CUDA;     \
+    } while (0)
+
+#define SP_LAUNCH_CHECK() SP_CUDA(cudaGetLastError())
+
+static inline int64_t sp_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// ---------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+__device__ __forceinline__ uint64_t sp_load_uint(const void* base, int64_t i, bool is64) {
+    return is64 ? static_cast<const uint64_t*>(base)[i] : static_cast<const uint32_t*>(base)[i];
+}
+__device__ __forceinline__ void sp_store_uint(void* base, int64_t i, uint64_t v, bool is64) {
+    if (is64) static_cast<uint64_t*>(base)[i] = v;
+    else static_cast<uint32_t*>(base)[i] = static_cast<uint32_t>(v);
+}
+
+__device__ __forceinline__ unsigned sp_lane() { return threadIdx.x & 31u; }
+
+__device__ __forceinline__ double sp_shfl(double v, int src) {
+    return __shfl_sync(0xffffffffu, v, src);
+}
+
+#endif  // __CUDACC__
+
+// Calls f(P{}, I{}) with the unsigned types matching the handle's widths.
+#define SP_DISPATCH_WIDTHS(t, ...)                                              \
+    do {                                                                        \
+        if ((t)->posBits == 32 && (t)->crdBits == 32) { using P = uint32_t; using I = uint32_t; __VA_ARGS__ } \
+        else if ((t)->posBits == 32) { using P = uint32_t; using I = uint64_t; __VA_ARGS__ }                 \
+        else if ((t)->crdBits == 32) { using P = uint64_t; using I = uint32_t; __VA_ARGS__ }                 \
+        else { using P = uint64_t; using I = uint64_t; __VA_ARGS__ }                                        \
+    } while (0)
+
+// Partition tables (partition.cu).  kind distinguishes the position array used.
+enum { SP_PART_MERGE_LAST = 1, SP_PART_MTTKRP = 2 };
+sp_status sp_get_merge_partition(sp_tensor* t, int64_t items_per_chunk, int64_t carry_elems_per_chunk,
+                                 cudaStream_t stream, sp_partition* out);
+sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t nnz_per_chunk, cudaStream_t stream, sp_partition* out);

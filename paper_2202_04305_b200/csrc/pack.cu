@@ -1,0 +1,743 @@
+// sp_pack / sp_unpack: coordinate list <-> per-level storage (Section 4.1 scheme,
+// reached through coordinates as in Section 4.2).
+//
+// Pipeline of sp_pack, all on the caller's stream:
+//   1. k_build_keys   level coordinates c_l = coord[dimOrdering[l]] fused into one
+//                     lexicographic key (level 0 in the top bits), range check
+//   2. radix sort     stable LSD, <= 8 bits per pass, (key, entry index) pairs;
+//                     per pass: tile histograms -> per-digit scan -> ranked scatter
+//   3. k_count_flags  for every level the flag "key prefix through this level
+//                     differs from the previous entry" = a new stored node;
+//                     per-tile counts, then a scan of the tile counts
+//   4. (one read-back of the node counts: the array sizes depend on the data)
+//   5. k_emit         node ids from the scanned flags; coordinates per node;
+//                     first-child offsets per parent; values (duplicates summed
+//                     in input order)
+//   6. suffix-min     compressed levels under a dense level: parents without
+//                     children take the next parent's offset
+#include "common.cuh"
+
+#include <string.h>
+
+namespace {
+
+constexpr int kErrRange = 1;
+constexpr int kErrDup = 2;
+
+struct LevelPlan {
+    int rank;
+    int shift[SP_MAX_RANK];
+    int bits[SP_MAX_RANK];
+    int lt[SP_MAX_RANK];
+    int src[SP_MAX_RANK];       // logical dimension stored at level l
+    int64_t sz[SP_MAX_RANK];
+};
+
+// ------------------------------------------------------------------ keys ---
+template <typename CT>
+__global__ void k_build_keys(const CT* c0, const CT* c1, const CT* c2, int64_t n, LevelPlan p,
+                             uint64_t* keys, uint32_t* idx, int* err) {
+    int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (e >= n) return;
+    const CT* src[SP_MAX_RANK] = {c0, c1, c2};
+    uint64_t key = 0;
+    bool bad = false;
+#pragma unroll
+    for (int l = 0; l < SP_MAX_RANK; ++l) {
+        if (l < p.rank) {
+            CT c = src[p.src[l]][e];
+            if (c < 0 || (int64_t)c >= p.sz[l]) { bad = true; c = 0; }
+            key |= (uint64_t)c << p.shift[l];
+        }
+    }
+    if (bad) atomicOr(err, kErrRange);
+    keys[e] = key;
+    idx[e] = (uint32_t)e;
+}
+
+// ------------------------------------------------------------ radix sort ---
+constexpr int kSortThreads = 256;
+constexpr int kSortIpt = 16;
+constexpr int kSortTile = kSortThreads * kSortIpt;   // 4096
+constexpr int kRadix = 256;
+constexpr int kSortWarps = kSortThreads / 32;
+
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint32_t u = __shfl_up_sync(0xffffffffu, v, o);
+        if ((int)sp_lane() >= o) v += u;
+    }
+    return v;
+}
+
+// Exclusive scan over the 256 threads of a block; `sums` has 8 entries.
+__device__ __forceinline__ uint32_t block256_excl_scan(uint32_t v, uint32_t* sums, uint32_t* total) {
+    const int w = threadIdx.x >> 5;
+    uint32_t incl = warp_incl_scan(v);
+    if (sp_lane() == 31) sums[w] = incl;
+    __syncthreads();
+    uint32_t pre = 0, tot = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        uint32_t s = sums[i];
+        if (i < w) pre += s;
+        tot += s;
+    }
+    __syncthreads();
+    *total = tot;
+    return incl - v + pre;
+}
+
+__global__ void __launch_bounds__(kSortThreads)
+k_sort_upsweep(const uint64_t* __restrict__ keys, int64_t n, int shift, uint32_t mask,
+               uint32_t* __restrict__ tilehist, int64_t ntiles) {
+    __shared__ uint32_t hist[kRadix];
+    const int t = threadIdx.x;
+    hist[t] = 0;
+    __syncthreads();
+    const int64_t base = (int64_t)blockIdx.x * kSortTile;
+#pragma unroll 4
+    for (int i = 0; i < kSortIpt; ++i) {
+        int64_t e = base + (int64_t)i * kSortThreads + t;
+        bool valid = e < n;
+        uint32_t d = valid ? ((uint32_t)(keys[e] >> shift) & mask) : (uint32_t)kRadix;
+        uint32_t peers = __match_any_sync(0xffffffffu, d);
+        if (valid && (int)sp_lane() == __ffs(peers) - 1) atomicAdd(&hist[d], (uint32_t)__popc(peers));
+    }
+    __syncthreads();
+    tilehist[(int64_t)t * ntiles + blockIdx.x] = hist[t];
+}
+
+// One block per digit: exclusive scan of that digit's tile counts, in place.
+__global__ void __launch_bounds__(256)
+k_sort_scan(uint32_t* tilehist, int64_t ntiles, uint32_t* digit_total) {
+    __shared__ uint32_t sums[8];
+    uint32_t* row = tilehist + (int64_t)blockIdx.x * ntiles;
+    uint32_t carry = 0;
+    for (int64_t base = 0; base < ntiles; base += 256) {
+        int64_t i = base + threadIdx.x;
+        uint32_t v = i < ntiles ? row[i] : 0u;
+        uint32_t tot;
+        uint32_t ex = block256_excl_scan(v, sums, &tot);
+        if (i < ntiles) row[i] = ex + carry;
+        carry += tot;
+    }
+    if (threadIdx.x == 0) digit_total[blockIdx.x] = carry;
+}
+
+constexpr size_t kDownSmem = (size_t)kSortTile * 8 + (size_t)kSortTile * 4 +
+                             (size_t)kSortWarps * (kRadix + 1) * 4 + (size_t)(kRadix + 1) * 4 + (size_t)kRadix * 8 + 64;
+
+__global__ void __launch_bounds__(kSortThreads)
+k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict__ idx_in,
+                 uint64_t* __restrict__ keys_out, uint32_t* __restrict__ idx_out, int64_t n, int shift,
+                 uint32_t mask, const uint32_t* __restrict__ tilehist, int64_t ntiles,
+                 const uint32_t* __restrict__ digit_total) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint64_t* skeys = reinterpret_cast<uint64_t*>(smem_raw);
+    uint32_t* sidx = reinterpret_cast<uint32_t*>(skeys + kSortTile);
+    uint32_t* wcnt = sidx + kSortTile;                       // [warps][kRadix + 1]
+    uint32_t* dstart = wcnt + kSortWarps * (kRadix + 1);      // [kRadix + 1]
+    int64_t* goff = reinterpret_cast<int64_t*>(dstart + (kRadix + 1) + 1);   // [kRadix], 8-byte aligned
+    __shared__ uint32_t sums[8];
+
+    const int t = threadIdx.x, w = t >> 5, lane = t & 31;
+    const int64_t base = (int64_t)blockIdx.x * kSortTile;
+    const int tile_n = (int)min((int64_t)kSortTile, n - base);
+
+    for (int i = t; i < kSortWarps * (kRadix + 1); i += kSortThreads) wcnt[i] = 0;
+    __syncthreads();
+
+    uint64_t key[kSortIpt];
+    uint32_t pay[kSortIpt];
+    uint32_t rank[kSortIpt];
+    uint32_t* mycnt = wcnt + w * (kRadix + 1);
+    const uint32_t lt_mask = (1u << lane) - 1u;
+#pragma unroll
+    for (int i = 0; i < kSortIpt; ++i) {
+        int li = w * (32 * kSortIpt) + i * 32 + lane;
+        bool valid = li < tile_n;
+        key[i] = valid ? keys_in[base + li] : 0;
+        pay[i] = valid ? idx_in[base + li] : 0;
+        uint32_t d = valid ? ((uint32_t)(key[i] >> shift) & mask) : (uint32_t)kRadix;
+        uint32_t peers = __match_any_sync(0xffffffffu, d);
+        int leader = __ffs(peers) - 1;
+        uint32_t b = 0;
+        if (lane == leader) { b = mycnt[d]; mycnt[d] = b + (uint32_t)__popc(peers); }
+        b = __shfl_sync(0xffffffffu, b, leader);
+        rank[i] = b + (uint32_t)__popc(peers & lt_mask);
+        __syncwarp();
+    }
+    __syncthreads();
+
+    // per digit: exclusive scan over warps; then exclusive scan over digits
+    uint32_t total = 0;
+    {
+        uint32_t run = 0;
+        for (int ww = 0; ww < kSortWarps; ++ww) {
+            uint32_t c = wcnt[ww * (kRadix + 1) + t];
+            wcnt[ww * (kRadix + 1) + t] = run;
+            run += c;
+        }
+        total = run;
+        if (t == 0) {   // the padding bin: invalid items sort after every real digit
+            uint32_t r2 = 0;
+            for (int ww = 0; ww < kSortWarps; ++ww) {
+                uint32_t c = wcnt[ww * (kRadix + 1) + kRadix];
+                wcnt[ww * (kRadix + 1) + kRadix] = r2;
+                r2 += c;
+            }
+        }
+    }
+    uint32_t tot_all;
+    uint32_t ex = block256_excl_scan(total, sums, &tot_all);
+    dstart[t] = ex;
+    if (t == 0) dstart[kRadix] = tot_all;
+    // global base of digit t = sum of totals of smaller digits + this tile's prefix within the digit
+    uint32_t dt = digit_total[t];
+    uint32_t gtot;
+    uint32_t gex = block256_excl_scan(dt, sums, &gtot);
+    goff[t] = (int64_t)gex + (int64_t)tilehist[(int64_t)t * ntiles + blockIdx.x] - (int64_t)ex;
+    __syncthreads();
+
+#pragma unroll
+    for (int i = 0; i < kSortIpt; ++i) {
+        int li = w * (32 * kSortIpt) + i * 32 + lane;
+        bool valid = li < tile_n;
+        uint32_t d = valid ? ((uint32_t)(key[i] >> shift) & mask) : (uint32_t)kRadix;
+        uint32_t s = dstart[d] + mycnt[d] + rank[i];
+        if (valid) { skeys[s] = key[i]; sidx[s] = pay[i]; }
+    }
+    __syncthreads();
+    for (int s = t; s < tile_n; s += kSortThreads) {
+        uint64_t k = skeys[s];
+        uint32_t d = (uint32_t)(k >> shift) & mask;
+        int64_t o = goff[d] + s;
+        keys_out[o] = k;
+        idx_out[o] = sidx[s];
+    }
+}
+
+// ------------------------------------------------- flags, counts, emit ---
+constexpr int kCtThreads = 256;
+constexpr int kCtIpt = 8;
+constexpr int kCtTile = kCtThreads * kCtIpt;   // 2048
+constexpr int kField = 21;                     // three 21-bit counters packed in 64 bits
+constexpr uint64_t kFieldMask = (1ull << kField) - 1;
+
+__device__ __forceinline__ uint64_t level_flags(uint64_t k, uint64_t kprev, bool first, const LevelPlan& p) {
+    uint64_t x = k ^ kprev, f = 0;
+#pragma unroll
+    for (int l = 0; l < SP_MAX_RANK; ++l)
+        if (l < p.rank) f |= (uint64_t)(first || (x >> p.shift[l]) != 0) << (kField * l);
+    return f;
+}
+
+__device__ __forceinline__ uint64_t warp_incl_scan64(uint64_t v) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint64_t u = __shfl_up_sync(0xffffffffu, v, o);
+        if ((int)sp_lane() >= o) v += u;
+    }
+    return v;
+}
+
+// Exclusive scan of packed counters over a block of up to 512 threads.
+__device__ __forceinline__ uint64_t block_excl_scan64(uint64_t v, uint64_t* sums, uint64_t* total) {
+    const int w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    uint64_t incl = warp_incl_scan64(v);
+    if (sp_lane() == 31) sums[w] = incl;
+    __syncthreads();
+    uint64_t pre = 0, tot = 0;
+    for (int i = 0; i < nw; ++i) {
+        uint64_t s = sums[i];
+        if (i < w) pre += s;
+        tot += s;
+    }
+    __syncthreads();
+    *total = tot;
+    return incl - v + pre;
+}
+
+__global__ void __launch_bounds__(kCtThreads)
+k_count_flags(const uint64_t* __restrict__ keys, int64_t n, LevelPlan p, uint64_t* __restrict__ tilesum) {
+    __shared__ uint64_t sums[16];
+    const int64_t e0 = (int64_t)blockIdx.x * kCtTile + (int64_t)threadIdx.x * kCtIpt;
+    uint64_t kprev = (e0 > 0 && e0 <= n) ? keys[e0 - 1] : 0;
+    uint64_t local = 0;
+#pragma unroll
+    for (int i = 0; i < kCtIpt; ++i) {
+        int64_t e = e0 + i;
+        if (e < n) {
+            uint64_t k = keys[e];
+            local += level_flags(k, kprev, e == 0, p);
+            kprev = k;
+        }
+    }
+    uint64_t tot;
+    block_excl_scan64(local, sums, &tot);
+    if (threadIdx.x == 0) tilesum[blockIdx.x] = tot;
+}
+
+// Single block (512 threads): tilesum (packed) -> tileprefix[l][tile] (exclusive), counts[l].
+__global__ void __launch_bounds__(512)
+k_scan_tiles(const uint64_t* __restrict__ tilesum, int64_t ntiles, int64_t* __restrict__ tileprefix,
+             int64_t* __restrict__ counts) {
+    __shared__ uint64_t sums[16];
+    int64_t run[SP_MAX_RANK] = {0, 0, 0};
+    for (int64_t base = 0; base < ntiles; base += 512) {
+        int64_t i = base + threadIdx.x;
+        uint64_t v = i < ntiles ? tilesum[i] : 0;
+        uint64_t tot;
+        uint64_t ex = block_excl_scan64(v, sums, &tot);
+#pragma unroll
+        for (int l = 0; l < SP_MAX_RANK; ++l) {
+            if (i < ntiles) tileprefix[(int64_t)l * ntiles + i] = run[l] + (int64_t)((ex >> (kField * l)) & kFieldMask);
+            run[l] += (int64_t)((tot >> (kField * l)) & kFieldMask);
+        }
+    }
+    if (threadIdx.x == 0)
+        for (int l = 0; l < SP_MAX_RANK; ++l) counts[l] = run[l];
+}
+
+struct EmitArgs {
+    const uint64_t* keys;
+    const uint32_t* idx;
+    const double* vals_in;
+    int64_t n;
+    LevelPlan plan;
+    const int64_t* tileprefix;
+    int64_t ntiles;
+    void* pos[SP_MAX_RANK];
+    void* crd[SP_MAX_RANK];
+    double* val;
+    bool pos64, crd64;
+    unsigned flags;
+    int* err;
+};
+
+__global__ void __launch_bounds__(kCtThreads) k_emit(EmitArgs a) {
+    __shared__ uint64_t sums[16];
+    const LevelPlan& p = a.plan;
+    const int64_t e0 = (int64_t)blockIdx.x * kCtTile + (int64_t)threadIdx.x * kCtIpt;
+    uint64_t k[kCtIpt], f[kCtIpt];
+    uint64_t kprev = (e0 > 0 && e0 <= a.n) ? a.keys[e0 - 1] : 0;
+    uint64_t local = 0;
+    {
+        uint64_t kp = kprev;
+#pragma unroll
+        for (int i = 0; i < kCtIpt; ++i) {
+            int64_t e = e0 + i;
+            k[i] = 0; f[i] = 0;
+            if (e < a.n) {
+                k[i] = a.keys[e];
+                f[i] = level_flags(k[i], kp, e == 0, p);
+                local += f[i];
+                kp = k[i];
+            }
+        }
+    }
+    uint64_t tot;
+    uint64_t ex = block_excl_scan64(local, sums, &tot);
+    int64_t incl[SP_MAX_RANK];
+#pragma unroll
+    for (int l = 0; l < SP_MAX_RANK; ++l)
+        incl[l] = a.tileprefix[(int64_t)l * a.ntiles + blockIdx.x] + (int64_t)((ex >> (kField * l)) & kFieldMask);
+
+    uint64_t kp = kprev;
+#pragma unroll
+    for (int i = 0; i < kCtIpt; ++i) {
+        int64_t e = e0 + i;
+        if (e >= a.n) break;
+        int64_t ppos = 0, pprev = 0;
+        bool full = false;
+#pragma unroll
+        for (int l = 0; l < SP_MAX_RANK; ++l) {
+            if (l >= p.rank) continue;
+            const uint64_t mask = p.bits[l] >= 64 ? ~0ull : ((1ull << p.bits[l]) - 1);
+            const int64_t c = (int64_t)((k[i] >> p.shift[l]) & mask);
+            const int64_t cp = (int64_t)((kp >> p.shift[l]) & mask);
+            const bool fl = (f[i] >> (kField * l)) & 1;
+            incl[l] += fl;
+            if (l == p.rank - 1) full = fl;
+            if (p.lt[l] == SP_DENSE) {
+                ppos = ppos * p.sz[l] + c;
+                pprev = pprev * p.sz[l] + cp;
+            } else {
+                const int64_t nid = incl[l] - 1;
+                if (fl) {
+                    sp_store_uint(a.crd[l], nid, (uint64_t)c, a.crd64);
+                    if (e == 0 || pprev != ppos) sp_store_uint(a.pos[l], ppos, (uint64_t)nid, a.pos64);
+                }
+                pprev = nid - (fl ? 1 : 0);
+                ppos = nid;
+            }
+        }
+        if (full) {
+            double s = a.vals_in[a.idx[e]];
+            for (int64_t g = e + 1; g < a.n && a.keys[g] == k[i]; ++g) s += a.vals_in[a.idx[g]];
+            a.val[ppos] = s;
+        } else if (a.flags & SP_DUP_ERROR) {
+            atomicOr(a.err, kErrDup);
+        }
+        kp = k[i];
+    }
+}
+
+__global__ void k_store_one(void* base, int64_t i, uint64_t v, bool is64) { sp_store_uint(base, i, v, is64); }
+
+// --------------------------------------------- suffix-min fill of pos[] ---
+// a[i] <- min(a[i..L-1]).  Written as a forward scan over r = L-1-i.
+template <typename T>
+__device__ __forceinline__ T tmin(T a, T b) { return a < b ? a : b; }
+
+template <typename T>
+__device__ __forceinline__ T block_excl_minscan(T v, T* sums, T* total, T ident) {
+    const int w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    T incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        T u = __shfl_up_sync(0xffffffffu, incl, o);
+        if ((int)sp_lane() >= o) incl = tmin(incl, u);
+    }
+    T exw = __shfl_up_sync(0xffffffffu, incl, 1);
+    if (sp_lane() == 0) exw = ident;
+    if (sp_lane() == 31) sums[w] = incl;
+    __syncthreads();
+    T pre = ident, tot = ident;
+    for (int i = 0; i < nw; ++i) {
+        T s = sums[i];
+        if (i < w) pre = tmin(pre, s);
+        tot = tmin(tot, s);
+    }
+    __syncthreads();
+    *total = tot;
+    return tmin(pre, exw);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kCtThreads) k_rmin_reduce(const T* __restrict__ a, int64_t L, T* __restrict__ tilemin) {
+    __shared__ T sums[16];
+    const T ident = ~(T)0;
+    int64_t r0 = (int64_t)blockIdx.x * kCtTile + (int64_t)threadIdx.x * kCtIpt;
+    T m = ident;
+#pragma unroll
+    for (int i = 0; i < kCtIpt; ++i) {
+        int64_t r = r0 + i;
+        if (r < L) m = tmin(m, a[L - 1 - r]);
+    }
+    T tot;
+    block_excl_minscan<T>(m, sums, &tot, ident);
+    if (threadIdx.x == 0) tilemin[blockIdx.x] = tot;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(512) k_rmin_tiles(T* tilemin, int64_t ntiles) {
+    __shared__ T sums[16];
+    const T ident = ~(T)0;
+    T carry = ident;
+    for (int64_t base = 0; base < ntiles; base += 512) {
+        int64_t i = base + threadIdx.x;
+        T v = i < ntiles ? tilemin[i] : ident;
+        T tot;
+        T ex = block_excl_minscan<T>(v, sums, &tot, ident);
+        if (i < ntiles) tilemin[i] = tmin(ex, carry);
+        carry = tmin(carry, tot);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kCtThreads) k_rmin_apply(T* __restrict__ a, int64_t L, const T* __restrict__ tilecarry) {
+    __shared__ T sums[16];
+    const T ident = ~(T)0;
+    int64_t r0 = (int64_t)blockIdx.x * kCtTile + (int64_t)threadIdx.x * kCtIpt;
+    T v[kCtIpt];
+    T m = ident;
+#pragma unroll
+    for (int i = 0; i < kCtIpt; ++i) {
+        int64_t r = r0 + i;
+        v[i] = r < L ? a[L - 1 - r] : ident;
+        m = tmin(m, v[i]);
+    }
+    T tot;
+    T run = tmin(block_excl_minscan<T>(m, sums, &tot, ident), tilecarry[blockIdx.x]);
+#pragma unroll
+    for (int i = 0; i < kCtIpt; ++i) {
+        int64_t r = r0 + i;
+        run = tmin(run, v[i]);
+        if (r < L) a[L - 1 - r] = run;
+    }
+}
+
+template <typename T>
+sp_status suffix_min_inplace(void* a, int64_t L, cudaStream_t stream) {
+    if (L <= 0) return SP_OK;
+    int64_t ntiles = sp_ceil_div(L, kCtTile);
+    sp_workspace ws(stream);
+    T* tm = ws.get<T>((size_t)ntiles);
+    if (ws.failed) return SP_ERR_ALLOC;
+    k_rmin_reduce<T><<<(unsigned)ntiles, kCtThreads, 0, stream>>>(static_cast<const T*>(a), L, tm);
+    k_rmin_tiles<T><<<1, 512, 0, stream>>>(tm, ntiles);
+    k_rmin_apply<T><<<(unsigned)ntiles, kCtThreads, 0, stream>>>(static_cast<T*>(a), L, tm);
+    SP_LAUNCH_CHECK();
+    return SP_OK;
+}
+
+// ---------------------------------------------------------------- unpack ---
+struct UnpackArgs {
+    int rank;
+    int lt[SP_MAX_RANK], ord[SP_MAX_RANK];
+    int64_t sz[SP_MAX_RANK];
+    const void* pos[SP_MAX_RANK];
+    int64_t npos[SP_MAX_RANK];
+    const void* crd[SP_MAX_RANK];
+    const double* val;
+    int64_t nval;
+    bool pos64, crd64;
+    int64_t* out[SP_MAX_RANK];
+    double* vals_out;
+};
+
+__global__ void k_unpack(UnpackArgs a) {
+    int64_t q = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (q >= a.nval) return;
+    a.vals_out[q] = a.val[q];
+    int64_t p = q;
+    for (int l = a.rank - 1; l >= 0; --l) {
+        int64_t c;
+        if (a.lt[l] == SP_DENSE) {
+            c = p % a.sz[l];
+            p /= a.sz[l];
+        } else {
+            c = (int64_t)sp_load_uint(a.crd[l], p, a.crd64);
+            // parent = last index whose offset is <= p
+            int64_t lo = 0, hi = a.npos[l] - 1;   // answer in [0, npos-2]
+            while (hi - lo > 1) {
+                int64_t mid = (lo + hi) >> 1;
+                if ((int64_t)sp_load_uint(a.pos[l], mid, a.pos64) <= p) lo = mid; else hi = mid;
+            }
+            p = lo;
+        }
+        a.out[a.ord[l]][q] = c;
+    }
+}
+
+int ceil_log2(int64_t v) {   // bits needed for coordinates 0..v-1
+    int b = 0;
+    while (b < 63 && ((int64_t)1 << b) < v) ++b;
+    return b;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------
+extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const void* const* coo_coords,
+                             int coo_coord_bits, const double* coo_vals, const sp_level_type* dimLevelType,
+                             const int* dimOrdering, int posBits, int crdBits, unsigned flags, void* stream_,
+                             sp_tensor** out) {
+    if (!out) return SP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (rank < 1 || rank > SP_MAX_RANK || !dims || !dimLevelType || nnz < 0) return SP_ERR_INVALID_ARG;
+    if (nnz > 0 && (!coo_coords || !coo_vals)) return SP_ERR_INVALID_ARG;
+    if (coo_coord_bits != 32 && coo_coord_bits != 64) return SP_ERR_INVALID_ARG;
+    if (posBits == 0) posBits = 64;
+    if (crdBits == 0) crdBits = 64;
+    if ((posBits != 32 && posBits != 64) || (crdBits != 32 && crdBits != 64)) return SP_ERR_INVALID_ARG;
+    if (flags > SP_DUP_ERROR) return SP_ERR_INVALID_ARG;
+    if (nnz >= ((int64_t)1 << 32)) return SP_ERR_UNSUPPORTED;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    LevelPlan plan;
+    memset(&plan, 0, sizeof plan);
+    plan.rank = rank;
+    bool seen[SP_MAX_RANK] = {false, false, false};
+    int total_bits = 0;
+    for (int l = 0; l < rank; ++l) {
+        int d = dimOrdering ? dimOrdering[l] : l;
+        if (d < 0 || d >= rank || seen[d]) return SP_ERR_INVALID_ARG;
+        seen[d] = true;
+        if (dims[d] < 1) return SP_ERR_INVALID_ARG;
+        if (dimLevelType[l] != SP_DENSE && dimLevelType[l] != SP_COMPRESSED) return SP_ERR_INVALID_ARG;
+        if (nnz > 0 && !coo_coords[d]) return SP_ERR_INVALID_ARG;
+        plan.src[l] = d;
+        plan.sz[l] = dims[d];
+        plan.lt[l] = dimLevelType[l];
+        plan.bits[l] = ceil_log2(dims[d]);
+        total_bits += plan.bits[l];
+    }
+    if (total_bits > 63) return SP_ERR_UNSUPPORTED;
+    for (int l = 0, s = total_bits; l < rank; ++l) { s -= plan.bits[l]; plan.shift[l] = s; }
+
+    const uint64_t max_pos = posBits == 32 ? 0xffffffffull : ~0ull;
+    const uint64_t max_crd = crdBits == 32 ? 0xffffffffull : ~0ull;
+    for (int l = 0; l < rank; ++l)
+        if (plan.lt[l] == SP_COMPRESSED && (uint64_t)(plan.sz[l] - 1) > max_crd) return SP_ERR_WIDTH_OVERFLOW;
+
+    sp_workspace ws(stream);
+    const int64_t n = nnz;
+    int64_t counts[SP_MAX_RANK] = {0, 0, 0};
+    uint64_t* keys = nullptr;
+    uint32_t* idx = nullptr;
+    int64_t* tileprefix = nullptr;
+    int* d_err = nullptr;
+    int64_t ct_tiles = 0;
+
+    if (n > 0) {
+        uint64_t* kbuf[2] = {ws.get<uint64_t>((size_t)n), ws.get<uint64_t>((size_t)n)};
+        uint32_t* ibuf[2] = {ws.get<uint32_t>((size_t)n), ws.get<uint32_t>((size_t)n)};
+        d_err = ws.get<int>(1);
+        const int64_t stiles = sp_ceil_div(n, kSortTile);
+        uint32_t* tilehist = ws.get<uint32_t>((size_t)stiles * kRadix);
+        uint32_t* digit_total = ws.get<uint32_t>(kRadix);
+        ct_tiles = sp_ceil_div(n, kCtTile);
+        uint64_t* tilesum = ws.get<uint64_t>((size_t)ct_tiles);
+        tileprefix = ws.get<int64_t>((size_t)ct_tiles * SP_MAX_RANK);
+        int64_t* d_counts = ws.get<int64_t>(SP_MAX_RANK);
+        if (ws.failed) return SP_ERR_ALLOC;
+        SP_CUDA(cudaMemsetAsync(d_err, 0, sizeof(int), stream));
+
+        const void* c[SP_MAX_RANK] = {coo_coords[0], rank > 1 ? coo_coords[1] : coo_coords[0],
+                                      rank > 2 ? coo_coords[2] : coo_coords[0]};
+        const unsigned kb = (unsigned)sp_ceil_div(n, 256);
+        if (coo_coord_bits == 32)
+            k_build_keys<int32_t><<<kb, 256, 0, stream>>>((const int32_t*)c[0], (const int32_t*)c[1],
+                                                          (const int32_t*)c[2], n, plan, kbuf[0], ibuf[0], d_err);
+        else
+            k_build_keys<int64_t><<<kb, 256, 0, stream>>>((const int64_t*)c[0], (const int64_t*)c[1],
+                                                          (const int64_t*)c[2], n, plan, kbuf[0], ibuf[0], d_err);
+        SP_LAUNCH_CHECK();
+
+        static bool attr_set = false;
+        if (!attr_set) {
+            SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDownSmem));
+            attr_set = true;
+        }
+        const int npasses = (total_bits + 7) / 8;
+        const int per = npasses ? (total_bits + npasses - 1) / npasses : 0;
+        int cur = 0;
+        for (int ps = 0; ps < npasses; ++ps) {
+            const int shift = ps * per;
+            const int width = (shift + per <= total_bits) ? per : (total_bits - shift);
+            const uint32_t mask = (1u << width) - 1u;
+            k_sort_upsweep<<<(unsigned)stiles, kSortThreads, 0, stream>>>(kbuf[cur], n, shift, mask, tilehist, stiles);
+            k_sort_scan<<<kRadix, 256, 0, stream>>>(tilehist, stiles, digit_total);
+            k_sort_downsweep<<<(unsigned)stiles, kSortThreads, kDownSmem, stream>>>(
+                kbuf[cur], ibuf[cur], kbuf[cur ^ 1], ibuf[cur ^ 1], n, shift, mask, tilehist, stiles, digit_total);
+            SP_LAUNCH_CHECK();
+            cur ^= 1;
+        }
+        keys = kbuf[cur];
+        idx = ibuf[cur];
+
+        k_count_flags<<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum);
+        k_scan_tiles<<<1, 512, 0, stream>>>(tilesum, ct_tiles, tileprefix, d_counts);
+        SP_LAUNCH_CHECK();
+        int h_err = 0;
+        SP_CUDA(cudaMemcpyAsync(counts, d_counts, sizeof counts, cudaMemcpyDeviceToHost, stream));
+        SP_CUDA(cudaMemcpyAsync(&h_err, d_err, sizeof h_err, cudaMemcpyDeviceToHost, stream));
+        SP_CUDA(cudaStreamSynchronize(stream));
+        if (h_err & kErrRange) return SP_ERR_OUT_OF_RANGE;
+        if ((flags & SP_DUP_ERROR) && counts[rank - 1] != n) return SP_ERR_DUPLICATE;
+    }
+
+    // sizes of the level arrays
+    sp_tensor* t = new sp_tensor();
+    cudaGetDevice(&t->device);
+    t->rank = rank;
+    t->posBits = posBits;
+    t->crdBits = crdBits;
+    const size_t pw = posBits / 8, cw = crdBits / 8;
+    sp_status st = SP_OK;
+    int64_t parents = 1;
+    int64_t parents_at[SP_MAX_RANK] = {0, 0, 0};
+    for (int l = 0; l < rank && st == SP_OK; ++l) {
+        t->dims[l] = dims[l];
+        t->lt[l] = plan.lt[l];
+        t->ord[l] = plan.src[l];
+        parents_at[l] = parents;
+        if (plan.lt[l] == SP_DENSE) {
+            if (parents > 0 && plan.sz[l] > (((int64_t)1 << 62) / parents)) { st = SP_ERR_ALLOC; break; }
+            parents *= plan.sz[l];
+        } else {
+            if ((uint64_t)counts[l] > max_pos) { st = SP_ERR_WIDTH_OVERFLOW; break; }
+            t->npos[l] = parents + 1;
+            t->ncrd[l] = counts[l];
+            t->pos[l] = sp_dev_alloc((size_t)t->npos[l] * pw, stream);
+            t->crd[l] = sp_dev_alloc((size_t)(counts[l] ? counts[l] : 1) * cw, stream);
+            if (!t->pos[l] || !t->crd[l]) { st = SP_ERR_ALLOC; break; }
+            parents = counts[l];
+        }
+    }
+    if (st == SP_OK) {
+        t->nval = parents;
+        t->val = static_cast<double*>(sp_dev_alloc((size_t)(parents ? parents : 1) * sizeof(double), stream));
+        if (!t->val) st = SP_ERR_ALLOC;
+    }
+    if (st != SP_OK) { sp_free(t); return st; }
+
+    auto fail = [&](sp_status s) { sp_free(t); return s; };
+#define SP_CUDA_T(call) do { if ((call) != cudaSuccess) return fail(SP_ERR_CUDA); } while (0)
+
+    const bool trailing_dense = plan.lt[rank - 1] == SP_DENSE;
+    if (trailing_dense && t->nval > 0) SP_CUDA_T(cudaMemsetAsync(t->val, 0, (size_t)t->nval * sizeof(double), stream));
+    bool needs_fill[SP_MAX_RANK] = {false, false, false};
+    for (int l = 0; l < rank; ++l) {
+        if (plan.lt[l] != SP_COMPRESSED) continue;
+        needs_fill[l] = n > 0 && l >= 1 && plan.lt[l - 1] == SP_DENSE;
+        if (n == 0) SP_CUDA_T(cudaMemsetAsync(t->pos[l], 0, (size_t)t->npos[l] * pw, stream));
+        else if (needs_fill[l]) SP_CUDA_T(cudaMemsetAsync(t->pos[l], 0xFF, (size_t)t->npos[l] * pw, stream));
+    }
+    if (n > 0) {
+        EmitArgs a;
+        a.keys = keys; a.idx = idx; a.vals_in = coo_vals; a.n = n; a.plan = plan;
+        a.tileprefix = tileprefix; a.ntiles = ct_tiles;
+        for (int l = 0; l < SP_MAX_RANK; ++l) { a.pos[l] = t->pos[l]; a.crd[l] = t->crd[l]; }
+        a.val = t->val; a.pos64 = posBits == 64; a.crd64 = crdBits == 64; a.flags = flags; a.err = d_err;
+        k_emit<<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);
+        for (int l = 0; l < rank; ++l) {
+            if (plan.lt[l] != SP_COMPRESSED) continue;
+            k_store_one<<<1, 1, 0, stream>>>(t->pos[l], parents_at[l], (uint64_t)counts[l], posBits == 64);
+            if (needs_fill[l]) {
+                sp_status s2 = posBits == 64 ? suffix_min_inplace<uint64_t>(t->pos[l], t->npos[l], stream)
+                                             : suffix_min_inplace<uint32_t>(t->pos[l], t->npos[l], stream);
+                if (s2 != SP_OK) return fail(s2);
+            }
+        }
+        SP_CUDA_T(cudaGetLastError());
+        // the workspace is released below; with the default allocator cudaFree waits for the stream
+    }
+#undef SP_CUDA_T
+    *out = t;
+    return SP_OK;
+}
+
+extern "C" sp_status sp_unpack(const sp_tensor* t, void* const* coo_coords_out, double* vals_out,
+                               int64_t* nnz_out, void* stream_) {
+    if (!t || !coo_coords_out || !vals_out || !nnz_out) return SP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    UnpackArgs a;
+    memset(&a, 0, sizeof a);
+    a.rank = t->rank;
+    for (int l = 0; l < t->rank; ++l) {
+        if (!coo_coords_out[l]) return SP_ERR_INVALID_ARG;
+        a.lt[l] = t->lt[l];
+        a.ord[l] = t->ord[l];
+        a.sz[l] = t->dims[t->ord[l]];
+        a.pos[l] = t->pos[l];
+        a.npos[l] = t->npos[l];
+        a.crd[l] = t->crd[l];
+        a.out[l] = static_cast<int64_t*>(coo_coords_out[l]);
+    }
+    a.val = t->val;
+    a.nval = t->nval;
+    a.pos64 = t->posBits == 64;
+    a.crd64 = t->crdBits == 64;
+    a.vals_out = vals_out;
+    *nnz_out = t->nval;
+    if (t->nval > 0) {
+        k_unpack<<<(unsigned)sp_ceil_div(t->nval, 256), 256, 0, stream>>>(a);
+        SP_LAUNCH_CHECK();
+    }
+    return SP_OK;
+}

@@ -1,0 +1,116 @@
+// Work partitions cached in a handle.
+//
+// Merge-path partition over the innermost compressed level: the list of segment
+// ends pos[1..S] (S segments = rows of a CSR matrix, stored rows of DCSR, columns
+// of CSC ...) is merged with the list of entry indices 0..nnz-1; chunk w starts at
+// the point of that merge path lying on diagonal w * items.  Every chunk then owns
+// the same number of (segment end + entry) items whatever the row-length skew.
+#include "common.cuh"
+
+namespace {
+
+template <typename P>
+__global__ void k_merge_partition(const P* __restrict__ pos, int64_t nseg, int64_t nnz, int64_t items,
+                                  int64_t nchunks, int64_t* __restrict__ row, int64_t* __restrict__ nz) {
+    int64_t w = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (w > nchunks) return;
+    const int64_t total = nseg + nnz;
+    int64_t d = w * items;
+    if (d > total) d = total;
+    int64_t lo = d > nnz ? d - nnz : 0;
+    int64_t hi = d < nseg ? d : nseg;
+    while (lo < hi) {
+        int64_t mid = (lo + hi) >> 1;
+        // segment end `mid` precedes entry (d - mid - 1) when all its entries are consumed
+        if ((int64_t)pos[mid + 1] <= d - mid - 1) lo = mid + 1; else hi = mid;
+    }
+    row[w] = lo;
+    nz[w] = d - lo;
+}
+
+// MTTKRP: equal ranges of innermost entries; for each range start the fibre
+// (level-1 node) and slice (level-0 node or index) that contain it.
+template <typename P>
+__global__ void k_mttkrp_partition(const P* __restrict__ pos1, int64_t nslice, const P* __restrict__ pos2,
+                                   int64_t nfiber, int64_t nnz, int64_t per, int64_t nchunks,
+                                   int64_t* __restrict__ fiber, int64_t* __restrict__ nz, int64_t* __restrict__ slice) {
+    int64_t w = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (w > nchunks) return;
+    int64_t p = w * per;
+    if (p >= nnz) { nz[w] = nnz; fiber[w] = nfiber; slice[w] = nslice; return; }
+    int64_t lo = 0, hi = nfiber;            // last f with pos2[f] <= p
+    while (hi - lo > 1) { int64_t mid = (lo + hi) >> 1; if ((int64_t)pos2[mid] <= p) lo = mid; else hi = mid; }
+    const int64_t f = lo;
+    lo = 0; hi = nslice;                    // last s with pos1[s] <= f
+    while (hi - lo > 1) { int64_t mid = (lo + hi) >> 1; if ((int64_t)pos1[mid] <= f) lo = mid; else hi = mid; }
+    nz[w] = p; fiber[w] = f; slice[w] = lo;
+}
+
+}  // namespace
+
+sp_status sp_get_merge_partition(sp_tensor* t, int64_t items, int64_t carry_elems_per_chunk, cudaStream_t stream,
+                                 sp_partition* out) {
+    std::lock_guard<std::mutex> lock(t->mu);
+    const uint64_t key = ((uint64_t)SP_PART_MERGE_LAST << 56) | ((uint64_t)carry_elems_per_chunk << 32) | (uint64_t)items;
+    auto it = t->parts.find(key);
+    if (it != t->parts.end()) { *out = it->second; return SP_OK; }
+    const int last = t->rank - 1;
+    const int64_t nseg = t->npos[last] - 1;
+    const int64_t nnz = t->ncrd[last];
+    sp_partition p;
+    p.nchunks = sp_ceil_div(nseg + nnz, items);
+    if (p.nchunks < 1) p.nchunks = 1;
+    p.row = static_cast<int64_t*>(sp_dev_alloc((size_t)(p.nchunks + 1) * sizeof(int64_t), stream));
+    p.nz = static_cast<int64_t*>(sp_dev_alloc((size_t)(p.nchunks + 1) * sizeof(int64_t), stream));
+    p.carry_elems = p.nchunks * (carry_elems_per_chunk + 1);
+    // carry: per chunk `carry_elems_per_chunk` doubles, then one int64 row id per chunk
+    p.carry = static_cast<double*>(sp_dev_alloc((size_t)p.carry_elems * sizeof(double), stream));
+    if (!p.row || !p.nz || !p.carry) {
+        sp_dev_free(p.row, stream); sp_dev_free(p.nz, stream); sp_dev_free(p.carry, stream);
+        return SP_ERR_ALLOC;
+    }
+    const unsigned blocks = (unsigned)sp_ceil_div(p.nchunks + 1, 256);
+    if (t->posBits == 32)
+        k_merge_partition<uint32_t><<<blocks, 256, 0, stream>>>(static_cast<const uint32_t*>(t->pos[last]), nseg, nnz,
+                                                                 items, p.nchunks, p.row, p.nz);
+    else
+        k_merge_partition<uint64_t><<<blocks, 256, 0, stream>>>(static_cast<const uint64_t*>(t->pos[last]), nseg, nnz,
+                                                                 items, p.nchunks, p.row, p.nz);
+    SP_LAUNCH_CHECK();
+    t->parts[key] = p;
+    *out = p;
+    return SP_OK;
+}
+
+sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t per, cudaStream_t stream, sp_partition* out) {
+    std::lock_guard<std::mutex> lock(t->mu);
+    const uint64_t key = ((uint64_t)SP_PART_MTTKRP << 56) | (uint64_t)per;
+    auto it = t->parts.find(key);
+    if (it != t->parts.end()) { *out = it->second; return SP_OK; }
+    const int64_t nnz = t->ncrd[2];
+    const int64_t nfiber = t->ncrd[1];
+    const int64_t nslice = t->npos[1] - 1;
+    sp_partition p;
+    p.nchunks = sp_ceil_div(nnz, per);
+    if (p.nchunks < 1) p.nchunks = 1;
+    p.row = static_cast<int64_t*>(sp_dev_alloc((size_t)(p.nchunks + 1) * sizeof(int64_t), stream));
+    p.nz = static_cast<int64_t*>(sp_dev_alloc((size_t)(p.nchunks + 1) * sizeof(int64_t), stream));
+    p.aux = static_cast<int64_t*>(sp_dev_alloc((size_t)(p.nchunks + 1) * sizeof(int64_t), stream));
+    if (!p.row || !p.nz || !p.aux) {
+        sp_dev_free(p.row, stream); sp_dev_free(p.nz, stream); sp_dev_free(p.aux, stream);
+        return SP_ERR_ALLOC;
+    }
+    const unsigned blocks = (unsigned)sp_ceil_div(p.nchunks + 1, 256);
+    if (t->posBits == 32)
+        k_mttkrp_partition<uint32_t><<<blocks, 256, 0, stream>>>(
+            static_cast<const uint32_t*>(t->pos[1]), nslice, static_cast<const uint32_t*>(t->pos[2]), nfiber, nnz, per,
+            p.nchunks, p.row, p.nz, p.aux);
+    else
+        k_mttkrp_partition<uint64_t><<<blocks, 256, 0, stream>>>(
+            static_cast<const uint64_t*>(t->pos[1]), nslice, static_cast<const uint64_t*>(t->pos[2]), nfiber, nnz, per,
+            p.nchunks, p.row, p.nz, p.aux);
+    SP_LAUNCH_CHECK();
+    t->parts[key] = p;
+    *out = p;
+    return SP_OK;
+}

@@ -1,0 +1,178 @@
+// sp_sddmm: X[i,j] = S[i,j] * sum_k A[i,k] * B[k,j] over the stored (i,j) of S
+// (Section 6.2), S in (dense|compressed, compressed) row-major storage.
+//
+// Loop shape: for each stored row i, for each p in pos[1][q]..pos[1][q+1]:
+// j = crd[1][p]; x[p] = S.val[p] * dot(A[i,:], B[:,j]).  B is given K x n row-major,
+// so a column is K elements a whole row apart; it is transposed once per call into
+// a workspace so each entry reads one contiguous K-vector.  The (row end, entry)
+// merge path is cut into equal pieces, one per warp; a warp keeps A[i,:] in
+// registers across the entries of a row and reduces each dot product with shuffles.
+#include "common.cuh"
+
+namespace {
+
+constexpr int kSThreads = 256;
+constexpr int kSItems = 64;   // merge items per warp
+
+__global__ void __launch_bounds__(256)
+k_transpose(const double* __restrict__ B, int64_t ldb, int64_t K, int64_t n, double* __restrict__ Bt, int64_t ldt) {
+    __shared__ double tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
+    const int64_t j0 = (int64_t)blockIdx.x * 32, k0 = (int64_t)blockIdx.y * 32;
+#pragma unroll
+    for (int r = ty; r < 32; r += 8) {
+        int64_t k = k0 + r, j = j0 + tx;
+        tile[r][tx] = (k < K && j < n) ? B[k * ldb + j] : 0.0;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = ty; r < 32; r += 8) {
+        int64_t j = j0 + r, k = k0 + tx;
+        if (j < n && k < K) Bt[j * ldt + k] = tile[tx][r];
+    }
+}
+
+template <int V>
+__device__ __forceinline__ void ld2(const double* p, double* a) {
+    if (V == 2) { double2 q = *reinterpret_cast<const double2*>(p); a[0] = q.x; a[V - 1] = q.y; }
+    else a[0] = *p;
+}
+
+// NCH > 0: A[i,:] lives in NCH register chunks of 32*V columns (K <= NCH*32*V).
+// NCH == 0: any K, A is re-read (from L1) for every entry.
+template <typename P, typename I, int V, int NCH>
+__global__ void __launch_bounds__(kSThreads)
+k_sddmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ sval,
+        const I* __restrict__ outer, const double* __restrict__ A, int64_t lda, const double* __restrict__ Bt,
+        int64_t ldt, int64_t K, double* __restrict__ xv, const int64_t* __restrict__ prow,
+        const int64_t* __restrict__ pnz, int64_t nchunks) {
+    const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    if (w >= nchunks) return;
+    const int lane = threadIdx.x & 31;
+    const int64_t i0 = prow[w], j0 = pnz[w], i1 = prow[w + 1], j1 = pnz[w + 1];
+    if (j1 == j0) return;
+
+    constexpr int NA = NCH > 0 ? NCH : 1;
+    double a[NA][V];
+    bool a_ready = false;
+    int64_t row = i0, p = j0, rbase = i0, nzbase = j0;
+    int64_t E = (rbase + lane < i1) ? (int64_t)pos[rbase + lane + 1] : j1;
+    I c_l = (nzbase + lane < j1) ? crd[nzbase + lane] : (I)0;
+    double v_l = (nzbase + lane < j1) ? sval[nzbase + lane] : 0.0;
+    double res = 0.0;
+
+    while (true) {
+        const int64_t rend = row < i1 ? __shfl_sync(0xffffffffu, E, (int)(row - rbase)) : j1;
+        const double* arow = nullptr;
+        if (p < rend) {
+            arow = A + (outer ? (int64_t)outer[row] : row) * lda;
+            if (NCH > 0 && !a_ready) {
+#pragma unroll
+                for (int ch = 0; ch < NA; ++ch) {
+                    const int64_t kk = (int64_t)ch * 32 * V + lane * V;
+#pragma unroll
+                    for (int q = 0; q < V; ++q) a[ch][q] = 0.0;
+                    if (kk < K) ld2<V>(arow + kk, a[ch]);
+                }
+                a_ready = true;
+            }
+        }
+        while (p < rend) {
+            int off = (int)(p - nzbase);
+            if (off == 32) {
+                if (nzbase + lane < j1) xv[nzbase + lane] = v_l * res;
+                nzbase += 32;
+                c_l = (nzbase + lane < j1) ? crd[nzbase + lane] : (I)0;
+                v_l = (nzbase + lane < j1) ? sval[nzbase + lane] : 0.0;
+                off = 0;
+            }
+            const int cnt = (int)min(rend - p, (int64_t)(32 - off));
+            for (int t = 0; t < cnt; ++t) {
+                const int64_t j = (int64_t)__shfl_sync(0xffffffffu, c_l, off + t);
+                const double* brow = Bt + j * ldt;
+                double part = 0.0;
+                if (NCH > 0) {
+#pragma unroll
+                    for (int ch = 0; ch < NA; ++ch) {
+                        const int64_t kk = (int64_t)ch * 32 * V + lane * V;
+                        if (kk < K) {
+                            double b[V];
+                            ld2<V>(brow + kk, b);
+#pragma unroll
+                            for (int q = 0; q < V; ++q) part = fma(a[ch][q], b[q], part);
+                        }
+                    }
+                } else {
+                    for (int64_t kk = (int64_t)lane * V; kk < K; kk += 32 * V) {
+                        double b[V], aa[V];
+                        ld2<V>(brow + kk, b);
+                        ld2<V>(arow + kk, aa);
+#pragma unroll
+                        for (int q = 0; q < V; ++q) part = fma(aa[q], b[q], part);
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                if (lane == off + t) res = part;
+            }
+            p += cnt;
+        }
+        if (row >= i1) break;
+        ++row;
+        a_ready = false;
+        if (row - rbase == 32) {
+            rbase += 32;
+            E = (rbase + lane < i1) ? (int64_t)pos[rbase + lane + 1] : j1;
+        }
+    }
+    if (nzbase + lane < j1) xv[nzbase + lane] = v_l * res;
+}
+
+}  // namespace
+
+extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const double* B, int64_t ldb, int64_t K,
+                              double* x_vals, void* stream_) {
+    if (!S || !A || !B || K < 1 || lda < K) return SP_ERR_INVALID_ARG;
+    if (S->rank != 2 || S->lt[1] != SP_COMPRESSED || S->ord[0] != 0 || S->ord[1] != 1) return SP_ERR_UNSUPPORTED;
+    const int64_t n = S->dims[1];
+    if (ldb < n) return SP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int64_t nnz = S->ncrd[1];
+    if (nnz == 0) return SP_OK;
+    if (!x_vals) return SP_ERR_INVALID_ARG;
+    const bool dbl = S->lt[0] == SP_COMPRESSED;
+
+    sp_workspace ws(stream);
+    const int64_t ldt = (K + 1) & ~(int64_t)1;   // even, so rows stay 16-byte aligned
+    double* Bt = ws.get<double>((size_t)n * ldt);
+    if (ws.failed) return SP_ERR_ALLOC;
+    dim3 tg((unsigned)sp_ceil_div(n, 32), (unsigned)sp_ceil_div(K, 32));
+    k_transpose<<<tg, 256, 0, stream>>>(B, ldb, K, n, Bt, ldt);
+    SP_LAUNCH_CHECK();
+
+    sp_partition part;
+    sp_status st = sp_get_merge_partition(S, kSItems, 0, stream, &part);
+    if (st != SP_OK) return st;
+    const bool vec2 = (K % 2 == 0) && (lda % 2 == 0) && (reinterpret_cast<uintptr_t>(A) % 16 == 0) &&
+                      (reinterpret_cast<uintptr_t>(Bt) % 16 == 0);
+    const unsigned blocks = (unsigned)sp_ceil_div(part.nchunks * 32, kSThreads);
+#define SP_SDDMM_LAUNCH(V, NCH)                                                                                     \
+    k_sddmm<P, I, V, NCH><<<blocks, kSThreads, 0, stream>>>(pos, crd, S->val, outer, A, lda, Bt, ldt, K, x_vals,    \
+                                                            part.row, part.nz, part.nchunks)
+    SP_DISPATCH_WIDTHS(S, {
+        const P* pos = static_cast<const P*>(S->pos[1]);
+        const I* crd = static_cast<const I*>(S->crd[1]);
+        const I* outer = dbl ? static_cast<const I*>(S->crd[0]) : nullptr;
+        if (vec2) {
+            if (K <= 64) SP_SDDMM_LAUNCH(2, 1);
+            else if (K <= 128) SP_SDDMM_LAUNCH(2, 2);
+            else if (K <= 256) SP_SDDMM_LAUNCH(2, 4);
+            else SP_SDDMM_LAUNCH(2, 0);
+        } else {
+            SP_SDDMM_LAUNCH(1, 0);
+        }
+    });
+#undef SP_SDDMM_LAUNCH
+    SP_LAUNCH_CHECK();
+    return SP_OK;
+}

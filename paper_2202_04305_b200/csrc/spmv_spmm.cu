@@ -1,0 +1,342 @@
+// sp_spmv and sp_spmm over (dense|compressed, compressed) storage in either
+// dimension order (CSR, DCSR, CSC, DCSC).
+//
+// The loops are the ones the paper's sparsification yields for
+// x[i] = A[i,j] * b[j] (Section 6.2) and C[i,j] = A[i,k] * B[k,j] (Section 1):
+// an outer loop over the level-0 index (all of it, or the stored ones through
+// crd[0]) and an inner loop over pos[1][q] .. pos[1][q+1].  Here the two loops
+// are flattened into one merge path over (segment ends, entries) and cut into
+// equal pieces, so a piece costs the same whatever the row-length skew.
+//
+// Row-major encodings reduce into rows: pieces write the rows that end inside
+// them and hand the open last row to a fix-up pass as a carry (no atomics).
+// Column-major encodings scatter into the output with f64 atomic adds.
+#include "common.cuh"
+
+namespace {
+
+// ===================================================================== SpMV
+constexpr int kVThreads = 256;
+constexpr int kVIpt = 8;
+constexpr int kVTile = kVThreads * kVIpt;   // merge items per CTA
+
+template <typename P, typename I, bool SCATTER>
+__global__ void __launch_bounds__(kVThreads)
+k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
+       const I* __restrict__ outer, const double* __restrict__ x, double* __restrict__ y,
+       const int64_t* __restrict__ prow, const int64_t* __restrict__ pnz, int64_t nseg,
+       double* __restrict__ carry_val, int64_t* __restrict__ carry_row) {
+    __shared__ int s_end[kVTile + 1];
+    __shared__ double s_prod[kVTile];
+    __shared__ I s_dst[SCATTER ? kVTile : 1];
+    __shared__ double s_wv[kVThreads / 32];
+    __shared__ int s_wf[kVThreads / 32];
+
+    const int t = threadIdx.x;
+    const int64_t i0 = prow[blockIdx.x], j0 = pnz[blockIdx.x];
+    const int64_t i1 = prow[blockIdx.x + 1], j1 = pnz[blockIdx.x + 1];
+    const int nrows = (int)(i1 - i0), nnzs = (int)(j1 - j0);
+
+    for (int r = t; r < nrows; r += kVThreads) s_end[r] = (int)((int64_t)pos[i0 + r + 1] - j0);
+    for (int jj = t; jj < nnzs; jj += kVThreads) {
+        const I c = crd[j0 + jj];
+        const double v = val[j0 + jj];
+        if (SCATTER) { s_prod[jj] = v; s_dst[jj] = c; }
+        else s_prod[jj] = v * __ldg(x + c);
+    }
+    __syncthreads();
+
+    const int total = nrows + nnzs;
+    const int d0 = min(t * kVIpt, total), d1 = min(d0 + kVIpt, total);
+    int lo = max(0, d0 - nnzs), hi = min(d0, nrows);
+    while (lo < hi) {
+        int mid = (lo + hi) >> 1;
+        if (s_end[mid] <= d0 - mid - 1) lo = mid + 1; else hi = mid;
+    }
+    int ti = lo, tj = d0 - lo;
+
+    if (SCATTER) {
+        // segment = a column of A; every entry adds val * x[col] into y[row]
+        int64_t seg = i0 + ti;
+        double xc = seg < nseg ? x[outer ? (int64_t)outer[seg] : seg] : 0.0;
+        for (int s = d0; s < d1; ++s) {
+            if (ti < nrows && s_end[ti] <= tj) {
+                ++ti; ++seg;
+                xc = seg < nseg ? x[outer ? (int64_t)outer[seg] : seg] : 0.0;
+            } else {
+                atomicAdd(y + (int64_t)s_dst[tj], s_prod[tj] * xc);
+                ++tj;
+            }
+        }
+        return;
+    }
+
+    double run = 0.0, first_val = 0.0;
+    int first_row = -1;
+    for (int s = d0; s < d1; ++s) {
+        if (ti < nrows && s_end[ti] <= tj) {
+            if (first_row < 0) { first_row = ti; first_val = run; }
+            else {
+                const int64_t r = i0 + ti;
+                y[outer ? (int64_t)outer[r] : r] = run;
+            }
+            run = 0.0;
+            ++ti;
+        } else {
+            run += s_prod[tj];
+            ++tj;
+        }
+    }
+    // carry chain across threads: out = flag ? run : in + run
+    int f = first_row >= 0;
+    double v = run;
+    const int lane = t & 31, w = t >> 5;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int fu = __shfl_up_sync(0xffffffffu, f, o);
+        double vu = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) { if (!f) v += vu; f |= fu; }
+    }
+    int fe = __shfl_up_sync(0xffffffffu, f, 1);
+    double ve = __shfl_up_sync(0xffffffffu, v, 1);
+    if (lane == 0) { fe = 0; ve = 0.0; }
+    if (lane == 31) { s_wf[w] = f; s_wv[w] = v; }
+    __syncthreads();
+    int pf = 0;
+    double pv = 0.0;
+    for (int i = 0; i < w; ++i) {
+        if (s_wf[i]) { pf = 1; pv = s_wv[i]; } else pv += s_wv[i];
+    }
+    const double in = fe ? ve : pv + ve;
+    (void)pf;
+    if (first_row >= 0) {
+        const int64_t r = i0 + first_row;
+        y[outer ? (int64_t)outer[r] : r] = first_val + in;
+    }
+    if (t == kVThreads - 1) {
+        const double outv = (first_row >= 0) ? run : in + run;
+        carry_val[blockIdx.x] = outv;
+        carry_row[blockIdx.x] = (i1 < nseg && j1 > j0) ? i1 : -1;
+    }
+}
+
+template <typename I>
+__global__ void k_spmv_fixup(const double* __restrict__ carry_val, const int64_t* __restrict__ carry_row,
+                             int64_t ntiles, const I* __restrict__ outer, double* __restrict__ y) {
+    int64_t w = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (w >= ntiles) return;
+    const int64_t r = carry_row[w];
+    if (r < 0 || (w > 0 && carry_row[w - 1] == r)) return;
+    double s = 0.0;
+    for (int64_t u = w; u < ntiles && carry_row[u] == r; ++u) s += carry_val[u];
+    y[outer ? (int64_t)outer[r] : r] += s;
+}
+
+// ===================================================================== SpMM
+constexpr int kMThreads = 256;
+constexpr int kMItems = 128;   // merge items per warp
+
+template <int V> struct vec_t;
+template <> struct vec_t<1> { double a[1]; };
+template <> struct __align__(16) vec_t<2> { double a[2]; };
+
+template <int V>
+__device__ __forceinline__ vec_t<V> ld_vec(const double* p) {
+    vec_t<V> r;
+    if (V == 2) { double2 q = *reinterpret_cast<const double2*>(p); r.a[0] = q.x; r.a[V - 1] = q.y; }
+    else r.a[0] = *p;
+    return r;
+}
+template <int V>
+__device__ __forceinline__ void st_vec(double* p, const double* a) {
+    if (V == 2) *reinterpret_cast<double2*>(p) = make_double2(a[0], a[V - 1]);
+    else *p = a[0];
+}
+
+template <typename P, typename I, int V, bool SCATTER>
+__global__ void __launch_bounds__(kMThreads)
+k_spmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
+       const I* __restrict__ outer, const double* __restrict__ B, int64_t N, int64_t ldb,
+       double* __restrict__ C, int64_t ldc, const int64_t* __restrict__ prow, const int64_t* __restrict__ pnz,
+       int64_t nchunks, int64_t nseg, double* __restrict__ carry, int64_t* __restrict__ carry_row) {
+    const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    if (w >= nchunks) return;
+    const int lane = threadIdx.x & 31;
+    const int64_t i0 = prow[w], j0 = pnz[w], i1 = prow[w + 1], j1 = pnz[w + 1];
+    int64_t pstart = j0;
+
+    for (int64_t cbase = 0; cbase < N; cbase += 32 * V) {
+        const int64_t col = cbase + (int64_t)lane * V;
+        const bool on = col < N;
+        double acc[V];
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc[q] = 0.0;
+        int64_t row = i0, p = j0, rbase = i0, nzbase = j0;
+        pstart = j0;
+        int64_t E = (rbase + lane < i1) ? (int64_t)pos[rbase + lane + 1] : j1;
+        I c_l = (nzbase + lane < j1) ? crd[nzbase + lane] : (I)0;
+        double v_l = (nzbase + lane < j1) ? val[nzbase + lane] : 0.0;
+        vec_t<V> brow;
+#pragma unroll
+        for (int q = 0; q < V; ++q) brow.a[q] = 0.0;
+        if (SCATTER && on && row < nseg) brow = ld_vec<V>(B + (outer ? (int64_t)outer[row] : row) * ldb + col);
+
+        while (true) {
+            const int64_t rend = row < i1 ? __shfl_sync(0xffffffffu, E, (int)(row - rbase)) : j1;
+            while (p < rend) {
+                int off = (int)(p - nzbase);
+                if (off == 32) {
+                    nzbase += 32;
+                    c_l = (nzbase + lane < j1) ? crd[nzbase + lane] : (I)0;
+                    v_l = (nzbase + lane < j1) ? val[nzbase + lane] : 0.0;
+                    off = 0;
+                }
+                const int cnt = (int)min(rend - p, (int64_t)(32 - off));
+                for (int t = 0; t < cnt; t += 4) {
+                    vec_t<V> b[4];
+                    double vv[4];
+                    int64_t kk[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        vv[u] = 0.0;
+                        kk[u] = 0;
+#pragma unroll
+                        for (int q = 0; q < V; ++q) b[u].a[q] = 0.0;
+                        if (t + u < cnt) {
+                            kk[u] = (int64_t)__shfl_sync(0xffffffffu, c_l, off + t + u);
+                            vv[u] = __shfl_sync(0xffffffffu, v_l, off + t + u);
+                            if (!SCATTER && on) b[u] = ld_vec<V>(B + kk[u] * ldb + col);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (SCATTER) {
+                            if (t + u < cnt && on) {
+#pragma unroll
+                                for (int q = 0; q < V; ++q) atomicAdd(C + kk[u] * ldc + col + q, vv[u] * brow.a[q]);
+                            }
+                        } else {
+#pragma unroll
+                            for (int q = 0; q < V; ++q) acc[q] = fma(vv[u], b[u].a[q], acc[q]);
+                        }
+                    }
+                }
+                p += cnt;
+            }
+            if (row >= i1) break;
+            if (!SCATTER && on) st_vec<V>(C + (outer ? (int64_t)outer[row] : row) * ldc + col, acc);
+#pragma unroll
+            for (int q = 0; q < V; ++q) acc[q] = 0.0;
+            ++row;
+            pstart = p;
+            if (row - rbase == 32) {
+                rbase += 32;
+                E = (rbase + lane < i1) ? (int64_t)pos[rbase + lane + 1] : j1;
+            }
+            if (SCATTER && on && row < nseg) brow = ld_vec<V>(B + (outer ? (int64_t)outer[row] : row) * ldb + col);
+        }
+        if (!SCATTER && on && j1 > pstart) st_vec<V>(carry + w * N + col, acc);
+    }
+    if (!SCATTER && lane == 0) carry_row[w] = (j1 > pstart && i1 < nseg) ? i1 : -1;
+}
+
+template <typename I>
+__global__ void k_spmm_fixup(const double* __restrict__ carry, const int64_t* __restrict__ carry_row,
+                             int64_t nchunks, const I* __restrict__ outer, int64_t N, double* __restrict__ C,
+                             int64_t ldc) {
+    const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    if (w >= nchunks) return;
+    const int lane = threadIdx.x & 31;
+    const int64_t r = carry_row[w];
+    if (r < 0 || (w > 0 && carry_row[w - 1] == r)) return;
+    int64_t end = w + 1;
+    while (end < nchunks && carry_row[end] == r) ++end;
+    double* crow = C + (outer ? (int64_t)outer[r] : r) * ldc;
+    for (int64_t col = lane; col < N; col += 32) {
+        double s = 0.0;
+        for (int64_t u = w; u < end; ++u) s += carry[u * N + col];
+        crow[col] += s;
+    }
+}
+
+bool matrix_encoding_ok(const sp_tensor* A) {
+    return A && A->rank == 2 && A->lt[1] == SP_COMPRESSED &&
+           ((A->ord[0] == 0 && A->ord[1] == 1) || (A->ord[0] == 1 && A->ord[1] == 0));
+}
+
+}  // namespace
+
+extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* stream_) {
+    if (!A || !x || !y) return SP_ERR_INVALID_ARG;
+    if (!matrix_encoding_ok(A)) return SP_ERR_UNSUPPORTED;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const bool rowmajor = A->ord[0] == 0;
+    const bool dbl = A->lt[0] == SP_COMPRESSED;
+    const int64_t m = A->dims[0];
+    if (!rowmajor || dbl) SP_CUDA(cudaMemsetAsync(y, 0, (size_t)m * sizeof(double), stream));
+    const int64_t nseg = A->npos[1] - 1;
+    if (nseg <= 0) return SP_OK;
+    sp_partition part;
+    sp_status st = sp_get_merge_partition(A, kVTile, 1, stream, &part);
+    if (st != SP_OK) return st;
+    double* cval = part.carry;
+    int64_t* crow = reinterpret_cast<int64_t*>(part.carry + part.nchunks);
+    SP_DISPATCH_WIDTHS(A, {
+        const P* pos = static_cast<const P*>(A->pos[1]);
+        const I* crd = static_cast<const I*>(A->crd[1]);
+        const I* outer = dbl ? static_cast<const I*>(A->crd[0]) : nullptr;
+        if (rowmajor) {
+            k_spmv<P, I, false><<<(unsigned)part.nchunks, kVThreads, 0, stream>>>(pos, crd, A->val, outer, x, y, part.row,
+                                                                                  part.nz, nseg, cval, crow);
+            k_spmv_fixup<I><<<(unsigned)sp_ceil_div(part.nchunks, 256), 256, 0, stream>>>(cval, crow, part.nchunks, outer, y);
+        } else {
+            k_spmv<P, I, true><<<(unsigned)part.nchunks, kVThreads, 0, stream>>>(pos, crd, A->val, outer, x, y, part.row,
+                                                                                 part.nz, nseg, cval, crow);
+        }
+    });
+    SP_LAUNCH_CHECK();
+    return SP_OK;
+}
+
+extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t ldb, double* C, int64_t ldc,
+                             void* stream_) {
+    if (!A || !B || !C || N < 1 || ldb < N || ldc < N) return SP_ERR_INVALID_ARG;
+    if (!matrix_encoding_ok(A)) return SP_ERR_UNSUPPORTED;
+    if (N >= (1 << 20)) return SP_ERR_UNSUPPORTED;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const bool rowmajor = A->ord[0] == 0;
+    const bool dbl = A->lt[0] == SP_COMPRESSED;
+    const int64_t m = A->dims[0];
+    if (!rowmajor || dbl) {
+        if (ldc == N) SP_CUDA(cudaMemsetAsync(C, 0, (size_t)m * N * sizeof(double), stream));
+        else SP_CUDA(cudaMemset2DAsync(C, (size_t)ldc * sizeof(double), 0, (size_t)N * sizeof(double), (size_t)m, stream));
+    }
+    const int64_t nseg = A->npos[1] - 1;
+    if (nseg <= 0) return SP_OK;
+    sp_partition part;
+    sp_status st = sp_get_merge_partition(A, kMItems, N, stream, &part);
+    if (st != SP_OK) return st;
+    double* carry = part.carry;
+    int64_t* crow = reinterpret_cast<int64_t*>(part.carry + part.nchunks * N);
+    const bool vec2 = N > 32 && (N % 2 == 0) && (ldb % 2 == 0) && (ldc % 2 == 0) &&
+                      (reinterpret_cast<uintptr_t>(B) % 16 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0) &&
+                      (reinterpret_cast<uintptr_t>(carry) % 16 == 0);
+    const unsigned blocks = (unsigned)sp_ceil_div(part.nchunks * 32, kMThreads);
+#define SP_SPMM_LAUNCH(V, SC)                                                                                   \
+    k_spmm<P, I, V, SC><<<blocks, kMThreads, 0, stream>>>(pos, crd, A->val, outer, B, N, ldb, C, ldc, part.row, \
+                                                          part.nz, part.nchunks, nseg, carry, crow)
+    SP_DISPATCH_WIDTHS(A, {
+        const P* pos = static_cast<const P*>(A->pos[1]);
+        const I* crd = static_cast<const I*>(A->crd[1]);
+        const I* outer = dbl ? static_cast<const I*>(A->crd[0]) : nullptr;
+        if (rowmajor) {
+            if (vec2) SP_SPMM_LAUNCH(2, false); else SP_SPMM_LAUNCH(1, false);
+            k_spmm_fixup<I><<<blocks, kMThreads, 0, stream>>>(carry, crow, part.nchunks, outer, N, C, ldc);
+        } else {
+            if (vec2) SP_SPMM_LAUNCH(2, true); else SP_SPMM_LAUNCH(1, true);
+        }
+    });
+#undef SP_SPMM_LAUNCH
+    SP_LAUNCH_CHECK();
+    return SP_OK;
+}

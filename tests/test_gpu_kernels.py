@@ -1,0 +1,187 @@
+"""sp_spmv / sp_spmm / sp_sddmm / sp_mttkrp through the C ABI against the oracle.
+
+Tolerance: |gpu - oracle| <= 1e-12 * sum|a*b| for every output entry (entries whose
+bound is 0 must be exactly 0); integer-valued inputs must match bit for bit."""
+import numpy as np
+import pytest
+
+from gpu_util import MATRIX_ENCODINGS, assert_close, dev, sp, to_dev
+from paper_2202_04305_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+def _matrices():
+    yield "uniform", I.uniform_matrix(300, 257, 4000, seed=1)
+    yield "tiny", I.uniform_matrix(3, 4, 5, seed=2)
+    yield "empty", I.uniform_matrix(17, 9, 0, seed=3)
+    yield "one_entry", I.uniform_matrix(40, 40, 1, seed=4)
+    yield "powerlaw", I.config2(seed=5, n=3000)
+    yield "confined", I.config3(seed=6, n=1 << 13, nnz=30000)
+    yield "band", I.row_band_matrix(700, 9, seed=7)
+    n = 5000   # one row holds everything / one column holds everything
+    yield "one_row", I.Coo((64, n), [np.full(n, 37), np.arange(n)], I.uniform_pm1(8, 1, n))
+    yield "one_col", I.Coo((n, 64), [np.arange(n), np.full(n, 11)], I.uniform_pm1(9, 1, n))
+
+
+MATS = list(_matrices())
+
+
+@pytest.mark.parametrize("enc", list(MATRIX_ENCODINGS))
+@pytest.mark.parametrize("name,coo", MATS, ids=[m[0] for m in MATS])
+def test_spmv(oracle, enc, name, coo):
+    lt, od = MATRIX_ENCODINGS[enc]
+    coords, vals = to_dev(coo)
+    A = sp().sp_pack(coo.dims, coords, vals, lt, od)
+    x = I.uniform_pm1(11, 2, coo.dims[1])
+    y = sp().sp_spmv(A, dev(x)).cpu().numpy()
+    ref, bd = oracle.spmv(coo.dims[0], coo.coords[0], coo.coords[1], coo.vals, x)
+    assert_close(y, ref, bd, f"spmv {enc} {name}")
+
+
+@pytest.mark.parametrize("enc", list(MATRIX_ENCODINGS))
+@pytest.mark.parametrize("N", [1, 5, 32, 64, 70])
+@pytest.mark.parametrize("name,coo", MATS, ids=[m[0] for m in MATS])
+def test_spmm(oracle, enc, N, name, coo):
+    if N in (5, 70) and name not in ("uniform", "powerlaw", "one_row"):
+        pytest.skip("ragged widths are covered on three matrices")
+    lt, od = MATRIX_ENCODINGS[enc]
+    coords, vals = to_dev(coo)
+    A = sp().sp_pack(coo.dims, coords, vals, lt, od)
+    B = I.dense_operand(12, 3, coo.dims[1], N)
+    Cg = sp().sp_spmm(A, dev(B)).cpu().numpy()
+    ref, bd = oracle.spmm(coo.dims[0], coo.coords[0], coo.coords[1], coo.vals, B)
+    assert_close(Cg, ref, bd, f"spmm {enc} {name} N={N}")
+
+
+def test_spmm_strided_operands_and_wide_indices(oracle):
+    import torch
+    coo = I.config2(seed=3, n=2000)
+    B = I.dense_operand(1, 4, 2000, 48)
+    ref, bd = oracle.spmm(2000, coo.coords[0], coo.coords[1], coo.vals, B)
+    for pb, cb, cbits in [(64, 64, 64), (32, 64, 32), (64, 32, 64)]:
+        coords, vals = to_dev(coo, cbits)
+        for enc in MATRIX_ENCODINGS.values():
+            A = sp().sp_pack(coo.dims, coords, vals, enc[0], enc[1], pb, cb)
+            Bbig = torch.zeros((2000, 50), dtype=torch.float64, device="cuda")
+            Bbig[:, :48] = dev(B)
+            Cbig = torch.full((2000, 51), 7.0, dtype=torch.float64, device="cuda")
+            sp().sp_spmm(A, Bbig[:, :48], Cbig[:, :48])
+            assert_close(Cbig[:, :48].cpu().numpy(), ref, bd, "strided")
+            assert torch.all(Cbig[:, 48:] == 7.0)
+
+
+def test_results_do_not_depend_on_encoding(oracle):
+    # Section 5.2: the result is independent of the sparsity annotation, up to reassociation.
+    coo = I.uniform_matrix(500, 400, 9000, seed=21)
+    B = I.dense_operand(2, 5, 400, 16)
+    ref, bd = oracle.spmm(500, coo.coords[0], coo.coords[1], coo.vals, B)
+    coords, vals = to_dev(coo)
+    outs = []
+    for lt, od in MATRIX_ENCODINGS.values():
+        for pb in (32, 64):
+            A = sp().sp_pack(coo.dims, coords, vals, lt, od, pb, pb)
+            outs.append(sp().sp_spmm(A, dev(B)).cpu().numpy())
+    for o in outs:
+        assert_close(o, ref, bd)
+        assert np.all(np.abs(o - outs[0]) <= 2e-12 * bd)
+
+
+def test_exact_for_integer_inputs(oracle):
+    coo = I.config2(seed=4, n=1500, integer_values=True)
+    B = I.dense_operand(3, 6, 1500, 64, integer_values=True)
+    x = I.small_ints(3, 7, 1500)
+    ref, _ = oracle.spmm(1500, coo.coords[0], coo.coords[1], coo.vals, B)
+    yref, _ = oracle.spmv(1500, coo.coords[0], coo.coords[1], coo.vals, x)
+    coords, vals = to_dev(coo)
+    for lt, od in MATRIX_ENCODINGS.values():
+        A = sp().sp_pack(coo.dims, coords, vals, lt, od)
+        assert np.array_equal(sp().sp_spmm(A, dev(B)).cpu().numpy(), ref)
+        assert np.array_equal(sp().sp_spmv(A, dev(x)).cpu().numpy(), yref)
+
+
+def test_unsupported_encodings():
+    b = sp()
+    coo = I.uniform_matrix(20, 20, 50, seed=1)
+    coords, vals = to_dev(coo)
+    A = b.sp_pack(coo.dims, coords, vals, (1, 0))
+    with pytest.raises(b.SpError) as e:
+        b.sp_spmv(A, dev(np.ones(20)))
+    assert e.value.code == 2
+    S = b.sp_pack(coo.dims, coords, vals, (0, 1), (1, 0))
+    with pytest.raises(b.SpError) as e:
+        b.sp_sddmm(S, dev(np.ones((20, 4))), dev(np.ones((4, 20))))
+    assert e.value.code == 2
+
+
+# ------------------------------------------------------------------ SDDMM
+@pytest.mark.parametrize("lt", [(0, 1), (1, 1)])
+@pytest.mark.parametrize("K", [1, 5, 64, 128, 130, 256, 300])
+def test_sddmm(oracle, lt, K):
+    for name, coo in [("uniform", I.uniform_matrix(300, 257, 4000, seed=1)), ("confined", I.config3(seed=6, n=1 << 12, nnz=9000)),
+                      ("one_row", MATS[7][1]), ("empty", I.uniform_matrix(9, 9, 0, seed=1))]:
+        coords, vals = to_dev(coo)
+        S = sp().sp_pack(coo.dims, coords, vals, lt)
+        A = I.dense_operand(13, 8, coo.dims[0], K)
+        B = I.dense_operand(13, 9, K, coo.dims[1])
+        xg = sp().sp_sddmm(S, dev(A), dev(B)).cpu().numpy()
+        xe, be = oracle.sddmm(coo.coords[0], coo.coords[1], coo.vals, A, B)
+        ep = oracle.pack(coo.dims, coo.coords, coo.vals, lt).entry_pos
+        ref = np.empty_like(xe); bd = np.empty_like(be)
+        ref[ep] = xe; bd[ep] = be
+        assert_close(xg, ref, bd, f"sddmm {name} K={K}")
+
+
+def test_sddmm_exact_integers(oracle):
+    coo = I.uniform_matrix(200, 200, 3000, seed=2, integer_values=True)
+    A = I.dense_operand(1, 8, 200, 128, integer_values=True)
+    B = I.dense_operand(1, 9, 128, 200, integer_values=True)
+    coords, vals = to_dev(coo)
+    S = sp().sp_pack(coo.dims, coords, vals, (0, 1))
+    xe, _ = oracle.sddmm(coo.coords[0], coo.coords[1], coo.vals, A, B)
+    ref = np.empty_like(xe)
+    ref[oracle.pack(coo.dims, coo.coords, coo.vals, (0, 1)).entry_pos] = xe
+    assert np.array_equal(sp().sp_sddmm(S, dev(A), dev(B)).cpu().numpy(), ref)
+
+
+# ----------------------------------------------------------------- MTTKRP
+TENSOR_ENCODINGS = {"CSF": ((1, 1, 1), (0, 1, 2)), "DSS": ((0, 1, 1), (0, 1, 2)), "DSS-alt": ((0, 1, 1), (0, 2, 1)),
+                    "CSF-alt": ((1, 1, 1), (0, 2, 1))}
+
+
+def _tensors():
+    yield "zipf", I.config5(seed=3, dim=200, nnz=40000)
+    yield "uniform", I.uniform_tensor((50, 40, 30), 3000, seed=4)
+    yield "tiny", I.uniform_tensor((3, 3, 4), 5, seed=5)
+    yield "empty", I.uniform_tensor((6, 5, 4), 0, seed=6)
+    n = 6000
+    yield "one_slice", I.Coo((10, 80, 90), [np.full(n, 3), np.arange(n) // 90 % 80, np.arange(n) % 90], I.uniform_pm1(1, 2, n))
+    yield "one_fibre", I.Coo((10, 8, n), [np.full(n, 9), np.full(n, 2), np.arange(n)], I.uniform_pm1(1, 3, n))
+
+
+TENS = list(_tensors())
+
+
+@pytest.mark.parametrize("enc", list(TENSOR_ENCODINGS))
+@pytest.mark.parametrize("R", [1, 5, 32, 40])
+@pytest.mark.parametrize("name,coo", TENS, ids=[t[0] for t in TENS])
+def test_mttkrp(oracle, enc, R, name, coo):
+    lt, od = TENSOR_ENCODINGS[enc]
+    coords, vals = to_dev(coo)
+    T = sp().sp_pack(coo.dims, coords, vals, lt, od)
+    B = I.dense_operand(14, 10, coo.dims[1], R)
+    Cf = I.dense_operand(14, 11, coo.dims[2], R)
+    M = sp().sp_mttkrp(T, dev(B), dev(Cf)).cpu().numpy()
+    ref, bd = oracle.mttkrp(coo.dims[0], *coo.coords, coo.vals, B, Cf)
+    assert_close(M, ref, bd, f"mttkrp {enc} {name} R={R}")
+
+
+def test_mttkrp_exact_integers(oracle):
+    coo = I.config5(seed=7, dim=128, nnz=20000, integer_values=True)
+    B = I.dense_operand(2, 10, 128, 32, integer_values=True)
+    Cf = I.dense_operand(2, 11, 128, 32, integer_values=True)
+    ref, _ = oracle.mttkrp(128, *coo.coords, coo.vals, B, Cf)
+    coords, vals = to_dev(coo)
+    for lt, od in TENSOR_ENCODINGS.values():
+        T = sp().sp_pack(coo.dims, coords, vals, lt, od)
+        assert np.array_equal(sp().sp_mttkrp(T, dev(B), dev(Cf)).cpu().numpy(), ref)

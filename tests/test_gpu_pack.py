@@ -1,0 +1,136 @@
+"""sp_pack / sp_unpack against the oracle packer: bit-exact positions, coordinates, values."""
+import numpy as np
+import pytest
+
+from conftest import GOLDEN_FILES, check_invariants, load_golden
+from gpu_util import all_encodings, assert_storage_equal, dev, sp, to_dev, unsigned
+from paper_2202_04305_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+def _pack_both(oracle, coo, lt, od, pb=32, cb=32, cbits=32, flags=0):
+    coords, vals = to_dev(coo, cbits)
+    t = sp().sp_pack(coo.dims, coords, vals, lt, od, pb, cb, flags)
+    ref = oracle.pack(coo.dims, coo.coords, coo.vals, lt, od)
+    return t, ref
+
+
+@pytest.mark.parametrize("name", GOLDEN_FILES)
+def test_paper_examples(oracle, name):
+    g = load_golden(name)
+    coo = I.Coo(g["dims"], g["coords"], g["vals"])
+    for pb, cb in [(32, 32), (64, 64), (0, 32)]:
+        t, _ = _pack_both(oracle, coo, g["lt"], g["ord"], pb, cb)
+        for l, tt in enumerate(g["lt"]):
+            if tt == 1:
+                assert np.array_equal(unsigned(t.positions(l)), g["pos"][l])
+                assert np.array_equal(unsigned(t.coordinates(l)), g["crd"][l])
+        assert np.array_equal(t.values().cpu().numpy(), g["val"])
+
+
+@pytest.mark.parametrize("dims,nnz", [((7,), 3), ((1,), 1), ((6, 5), 11), ((5, 8), 0), ((1, 9), 4), ((4, 3, 5), 17),
+                                      ((3, 3, 4), 36), ((40, 50, 60), 5000)])
+def test_every_encoding_small(oracle, dims, nnz):
+    coo = I.uniform_tensor(dims, nnz, seed=len(dims) * 100 + nnz)
+    for lt, od in all_encodings(len(dims)):
+        for pb, cb, cbits in [(32, 32, 32), (64, 64, 64)]:
+            t, ref = _pack_both(oracle, coo, lt, od, pb, cb, cbits)
+            assert_storage_equal(t, ref)
+            check_invariants(dims, lt, od, [unsigned(t.positions(l)) if lt[l] else None for l in range(len(dims))],
+                             [unsigned(t.coordinates(l)) if lt[l] else None for l in range(len(dims))],
+                             t.values().cpu().numpy())
+
+
+@pytest.mark.parametrize("m,n,nnz", [(1000, 900, 4096 * 3 + 17), (70000, 300, 100001), (5, 200000, 4097), (300000, 300000, 250000)])
+@pytest.mark.parametrize("enc", [((0, 1), (0, 1)), ((1, 1), (0, 1)), ((0, 1), (1, 0)), ((1, 1), (1, 0)), ((1, 0), (0, 1))])
+def test_matrices_spanning_tiles(oracle, m, n, nnz, enc):
+    lt, od = enc
+    if lt == (1, 0) and m * n > 1 << 26:
+        pytest.skip("dense inner level too large to materialise")
+    coo = I.uniform_matrix(m, n, nnz, seed=m % 97)
+    t, ref = _pack_both(oracle, coo, lt, od)
+    assert_storage_equal(t, ref)
+
+
+def test_confined_rows_and_power_law(oracle):
+    for coo in (I.config3(seed=1, n=1 << 14, nnz=60000), I.config2(seed=1, n=4096)):
+        for lt, od in [((0, 1), (0, 1)), ((1, 1), (0, 1)), ((0, 1), (1, 0))]:
+            t, ref = _pack_both(oracle, coo, lt, od)
+            assert_storage_equal(t, ref)
+
+
+@pytest.mark.parametrize("enc", [((1, 1, 1), (0, 1, 2)), ((0, 1, 1), (0, 1, 2)), ((0, 1, 1), (0, 2, 1)), ((1, 1, 1), (2, 0, 1)),
+                                 ((0, 0, 1), (1, 2, 0)), ((1, 0, 1), (0, 1, 2))])
+def test_zipf_tensor(oracle, enc):
+    coo = I.config5(seed=2, dim=256, nnz=70001)
+    t, ref = _pack_both(oracle, coo, *enc)
+    assert_storage_equal(t, ref)
+
+
+def test_duplicates_zeros_and_flags(oracle):
+    coo = I.uniform_matrix(50, 60, 500, seed=8)
+    coords = [np.concatenate([c, c[:100], c[50:80]]) for c in coo.coords]
+    vals = np.concatenate([coo.vals, I.uniform_pm1(8, 70, 130)])
+    vals[::7] = 0.0
+    dup = I.Coo(coo.dims, coords, vals)
+    for lt, od in [((0, 1), (0, 1)), ((1, 1), (1, 0)), ((1, 0), (0, 1))]:
+        t, ref = _pack_both(oracle, dup, lt, od)
+        assert_storage_equal(t, ref)          # same summation order => same bits
+    b = sp()
+    c, v = to_dev(dup)
+    with pytest.raises(b.SpError) as e:
+        b.sp_pack(dup.dims, c, v, (0, 1), None, 32, 32, b.DUP_ERROR)
+    assert e.value.code == 5
+    c, v = to_dev(coo)
+    b.sp_pack(coo.dims, c, v, (0, 1), None, 32, 32, b.DUP_ERROR)   # duplicate-free input passes
+
+
+def test_error_codes():
+    b = sp()
+    coo = I.uniform_matrix(10, 10, 20, seed=1)
+    c, v = to_dev(coo)
+    bad = [c[0].clone(), c[1].clone()]
+    bad[1][3] = 10
+    with pytest.raises(b.SpError) as e:
+        b.sp_pack(coo.dims, bad, v, (0, 1))
+    assert e.value.code == 3
+    bad[1][3] = -1
+    with pytest.raises(b.SpError) as e:
+        b.sp_pack(coo.dims, bad, v, (0, 1))
+    assert e.value.code == 3
+    with pytest.raises(b.SpError) as e:
+        b.sp_pack(coo.dims, c, v, (0, 1), (0, 0))
+    assert e.value.code == 1
+    with pytest.raises(b.SpError) as e:
+        b.sp_pack(coo.dims, c, v, (0, 1), None, 16, 32)
+    assert e.value.code == 1
+    with pytest.raises(b.SpError) as e:           # 2^33 columns do not fit 32-bit coordinates
+        b.sp_pack((4, 1 << 33), c, v, (0, 1), None, 32, 32)
+    assert e.value.code == 4
+    t = b.sp_pack((4, 1 << 33), [c[0] % 4, c[1]], v, (0, 1), None, 32, 64)
+    assert t.coordinates(1).dtype.itemsize == 8
+
+
+def test_unpack_round_trip(oracle):
+    for dims, nnz in [((30, 40), 333), ((9, 8, 7), 200)]:
+        coo = I.uniform_tensor(dims, nnz, seed=5)
+        for lt, od in all_encodings(len(dims)):
+            coords, vals = to_dev(coo)
+            t = sp().sp_pack(dims, coords, vals, lt, od)
+            oc, ov = sp().sp_unpack(t)
+            rc, rv = oracle.unpack(oracle.pack(dims, coo.coords, coo.vals, lt, od))
+            for d in range(len(dims)):
+                assert np.array_equal(oc[d].cpu().numpy(), rc[d])
+            assert np.array_equal(ov.cpu().numpy(), rv)
+
+
+def test_pack_is_repeatable():
+    coo = I.uniform_matrix(5000, 5000, 200000, seed=3)
+    coords, vals = to_dev(coo)
+    a = sp().sp_pack(coo.dims, coords, vals, (1, 1))
+    b = sp().sp_pack(coo.dims, coords, vals, (1, 1))
+    for l in range(2):
+        assert np.array_equal(a.positions(l).cpu().numpy(), b.positions(l).cpu().numpy())
+        assert np.array_equal(a.coordinates(l).cpu().numpy(), b.coordinates(l).cpu().numpy())
+    assert np.array_equal(a.values().cpu().numpy(), b.values().cpu().numpy())
