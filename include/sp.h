@@ -167,6 +167,20 @@ sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const double* B, 
 sp_status sp_mttkrp(sp_tensor* T, const double* B, const double* C, int64_t R,
                     double* M, void* stream);
 
+/*
+ * Measurement aids (no counterpart in the paper).
+ * sp_launch_count: number of kernels this library has launched in this process.
+ * sp_set_profiling(1): sp_pack brackets its phases with CUDA events on the caller's
+ * stream (this adds small gaps between its kernels; leave it off when timing calls).
+ * sp_get_pack_profile: milliseconds of the last profiled sp_pack per phase
+ * (ms has SP_PACK_PROFILE_LEN entries: key build, sort histograms, sort scans,
+ * sort scatters, node counting, emit + fill) and the number of sort passes.
+ */
+#define SP_PACK_PROFILE_LEN 6
+int64_t sp_launch_count(void);
+sp_status sp_set_profiling(int enabled);
+sp_status sp_get_pack_profile(double* ms /* host */, int* npasses /* host, may be NULL */);
+
 #ifdef __cplusplus
 }
 #endif

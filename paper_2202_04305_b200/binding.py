@@ -18,7 +18,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libsp.so")
 
 SYMBOLS = ["sp_status_string", "sp_set_allocator", "sp_pack", "sp_free", "sp_info", "sp_positions",
-           "sp_coordinates", "sp_values", "sp_unpack", "sp_spmv", "sp_spmm", "sp_sddmm", "sp_mttkrp"]
+           "sp_coordinates", "sp_values", "sp_unpack", "sp_spmv", "sp_spmm", "sp_sddmm", "sp_mttkrp",
+           "sp_set_profiling", "sp_get_pack_profile", "sp_launch_count"]
 
 
 class SpError(RuntimeError):
@@ -36,6 +37,7 @@ def _load():
     lib.sp_status_string.argtypes = [C.c_int]
     for name in SYMBOLS[1:]:
         getattr(lib, name).restype = C.c_int
+    lib.sp_launch_count.restype = C.c_int64
     return lib
 
 
@@ -226,3 +228,22 @@ def sp_mttkrp(T: SpTensor, B, Cf, M=None):
         M = torch.empty((T.dims[0], R), dtype=torch.float64, device="cuda")
     _check(_lib.sp_mttkrp(T._h, _dptr(B), _dptr(Cf), C.c_int64(R), _dptr(M), _stream()), "sp_mttkrp")
     return M
+
+
+def sp_launch_count() -> int:
+    return int(_lib.sp_launch_count())
+
+
+def sp_set_profiling(enabled: bool):
+    _check(_lib.sp_set_profiling(C.c_int(1 if enabled else 0)), "sp_set_profiling")
+
+
+PACK_PHASES = ("keys", "sort_hist", "sort_scan", "sort_scatter", "count", "emit")
+
+
+def sp_get_pack_profile():
+    """(dict phase -> ms, number of sort passes) of the last sp_pack run with profiling on."""
+    ms = (C.c_double * len(PACK_PHASES))()
+    n = C.c_int()
+    _check(_lib.sp_get_pack_profile(ms, C.byref(n)), "sp_get_pack_profile")
+    return {k: ms[i] for i, k in enumerate(PACK_PHASES)}, n.value

@@ -1,11 +1,16 @@
 // Handle management, allocator plumbing and the accessor calls of sp.h.
 #include "common.cuh"
 
+#include <atomic>
+
 namespace {
 void* (*g_alloc)(size_t, void*, void*) = nullptr;
 void (*g_dealloc)(void*, void*, void*) = nullptr;
 void* g_ctx = nullptr;
+std::atomic<int64_t> g_launches{0};
 }  // namespace
+
+void sp_count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 void* sp_dev_alloc(size_t bytes, cudaStream_t stream) {
     if (g_alloc) return g_alloc(bytes, stream, g_ctx);
@@ -21,6 +26,8 @@ void sp_dev_free(void* p, cudaStream_t stream) {
 }
 
 extern "C" {
+
+int64_t sp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* sp_status_string(sp_status s) {
     switch (s) {

@@ -70,6 +70,8 @@ struct sp_workspace {
     }
 };
 
+void sp_count_launches(int n);
+
 #define SP_CUDA(call)                                   \
     do {                                                \
         cudaError_t e__ = (call);                       \

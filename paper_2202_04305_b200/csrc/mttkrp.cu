@@ -124,5 +124,6 @@ extern "C" sp_status sp_mttkrp(sp_tensor* T, const double* B, const double* C, i
             T->val, F1, F2, R, M, part.row, part.nz, part.aux, part.nchunks, T->npos[1] - 1, T->ncrd[1]);
     });
     SP_LAUNCH_CHECK();
+    sp_count_launches(1);
     return SP_OK;
 }

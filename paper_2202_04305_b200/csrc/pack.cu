@@ -24,6 +24,41 @@ namespace {
 constexpr int kErrRange = 1;
 constexpr int kErrDup = 2;
 
+// Optional phase timing of sp_pack (sp_set_profiling): CUDA events on the caller's stream.
+enum { kPhKeys = 0, kPhUpsweep, kPhScan, kPhDownsweep, kPhCount, kPhEmit, kPhCount_ };
+bool g_profiling = false;
+double g_phase_ms[SP_PACK_PROFILE_LEN] = {0, 0, 0, 0, 0, 0};
+int g_phase_passes = 0;
+
+struct PhaseTimer {
+    cudaStream_t stream;
+    bool on;
+    std::vector<cudaEvent_t> ev;
+    std::vector<int> phase;
+    PhaseTimer(cudaStream_t s, bool enabled) : stream(s), on(enabled) { if (on) mark(-1); }
+    // closes the interval that started at the previous mark and files it under `ph`
+    void mark(int ph) {
+        if (!on) return;
+        cudaEvent_t e;
+        cudaEventCreate(&e);
+        cudaEventRecord(e, stream);
+        ev.push_back(e);
+        phase.push_back(ph);
+    }
+    void finish(int passes) {
+        if (!on) return;
+        cudaEventSynchronize(ev.back());
+        for (int i = 0; i < SP_PACK_PROFILE_LEN; ++i) g_phase_ms[i] = 0;
+        for (size_t i = 1; i < ev.size(); ++i) {
+            float ms = 0;
+            cudaEventElapsedTime(&ms, ev[i - 1], ev[i]);
+            if (phase[i] >= 0) g_phase_ms[phase[i]] += ms;
+        }
+        g_phase_passes = passes;
+    }
+    ~PhaseTimer() { for (auto e : ev) cudaEventDestroy(e); }
+};
+
 struct LevelPlan {
     int rank;
     int shift[SP_MAX_RANK];
@@ -480,6 +515,7 @@ sp_status suffix_min_inplace(void* a, int64_t L, cudaStream_t stream) {
     k_rmin_reduce<T><<<(unsigned)ntiles, kCtThreads, 0, stream>>>(static_cast<const T*>(a), L, tm);
     k_rmin_tiles<T><<<1, 512, 0, stream>>>(tm, ntiles);
     k_rmin_apply<T><<<(unsigned)ntiles, kCtThreads, 0, stream>>>(static_cast<T*>(a), L, tm);
+    sp_count_launches(3);
     SP_LAUNCH_CHECK();
     return SP_OK;
 }
@@ -575,6 +611,8 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
         if (plan.lt[l] == SP_COMPRESSED && (uint64_t)(plan.sz[l] - 1) > max_crd) return SP_ERR_WIDTH_OVERFLOW;
 
     sp_workspace ws(stream);
+    PhaseTimer timer(stream, g_profiling);
+    int npasses_done = 0;
     const int64_t n = nnz;
     int64_t counts[SP_MAX_RANK] = {0, 0, 0};
     uint64_t* keys = nullptr;
@@ -607,12 +645,9 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
             k_build_keys<int64_t><<<kb, 256, 0, stream>>>((const int64_t*)c[0], (const int64_t*)c[1],
                                                           (const int64_t*)c[2], n, plan, kbuf[0], ibuf[0], d_err);
         SP_LAUNCH_CHECK();
-
-        static bool attr_set = false;
-        if (!attr_set) {
-            SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDownSmem));
-            attr_set = true;
-        }
+        sp_count_launches(1);
+        timer.mark(kPhKeys);
+        SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDownSmem));
         const int npasses = (total_bits + 7) / 8;
         const int per = npasses ? (total_bits + npasses - 1) / npasses : 0;
         int cur = 0;
@@ -621,18 +656,25 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
             const int width = (shift + per <= total_bits) ? per : (total_bits - shift);
             const uint32_t mask = (1u << width) - 1u;
             k_sort_upsweep<<<(unsigned)stiles, kSortThreads, 0, stream>>>(kbuf[cur], n, shift, mask, tilehist, stiles);
+            timer.mark(kPhUpsweep);
             k_sort_scan<<<kRadix, 256, 0, stream>>>(tilehist, stiles, digit_total);
+            timer.mark(kPhScan);
             k_sort_downsweep<<<(unsigned)stiles, kSortThreads, kDownSmem, stream>>>(
                 kbuf[cur], ibuf[cur], kbuf[cur ^ 1], ibuf[cur ^ 1], n, shift, mask, tilehist, stiles, digit_total);
             SP_LAUNCH_CHECK();
+            timer.mark(kPhDownsweep);
+            sp_count_launches(3);
             cur ^= 1;
         }
+        npasses_done = npasses;
         keys = kbuf[cur];
         idx = ibuf[cur];
 
         k_count_flags<<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum);
         k_scan_tiles<<<1, 512, 0, stream>>>(tilesum, ct_tiles, tileprefix, d_counts);
         SP_LAUNCH_CHECK();
+        timer.mark(kPhCount);
+        sp_count_launches(3);
         int h_err = 0;
         SP_CUDA(cudaMemcpyAsync(counts, d_counts, sizeof counts, cudaMemcpyDeviceToHost, stream));
         SP_CUDA(cudaMemcpyAsync(&h_err, d_err, sizeof h_err, cudaMemcpyDeviceToHost, stream));
@@ -695,9 +737,11 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
         for (int l = 0; l < SP_MAX_RANK; ++l) { a.pos[l] = t->pos[l]; a.crd[l] = t->crd[l]; }
         a.val = t->val; a.pos64 = posBits == 64; a.crd64 = crdBits == 64; a.flags = flags; a.err = d_err;
         k_emit<<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);
+        sp_count_launches(1);
         for (int l = 0; l < rank; ++l) {
             if (plan.lt[l] != SP_COMPRESSED) continue;
             k_store_one<<<1, 1, 0, stream>>>(t->pos[l], parents_at[l], (uint64_t)counts[l], posBits == 64);
+            sp_count_launches(1);
             if (needs_fill[l]) {
                 sp_status s2 = posBits == 64 ? suffix_min_inplace<uint64_t>(t->pos[l], t->npos[l], stream)
                                              : suffix_min_inplace<uint32_t>(t->pos[l], t->npos[l], stream);
@@ -705,10 +749,24 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
             }
         }
         SP_CUDA_T(cudaGetLastError());
+        timer.mark(kPhEmit);
+        timer.finish(npasses_done);
         // the workspace is released below; with the default allocator cudaFree waits for the stream
     }
 #undef SP_CUDA_T
     *out = t;
+    return SP_OK;
+}
+
+extern "C" sp_status sp_set_profiling(int enabled) {
+    g_profiling = enabled != 0;
+    return SP_OK;
+}
+
+extern "C" sp_status sp_get_pack_profile(double* ms, int* npasses) {
+    if (!ms) return SP_ERR_INVALID_ARG;
+    for (int i = 0; i < SP_PACK_PROFILE_LEN; ++i) ms[i] = g_phase_ms[i];
+    if (npasses) *npasses = g_phase_passes;
     return SP_OK;
 }
 
@@ -737,6 +795,7 @@ extern "C" sp_status sp_unpack(const sp_tensor* t, void* const* coo_coords_out, 
     *nnz_out = t->nval;
     if (t->nval > 0) {
         k_unpack<<<(unsigned)sp_ceil_div(t->nval, 256), 256, 0, stream>>>(a);
+        sp_count_launches(1);
         SP_LAUNCH_CHECK();
     }
     return SP_OK;

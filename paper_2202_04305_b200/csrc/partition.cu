@@ -77,6 +77,7 @@ sp_status sp_get_merge_partition(sp_tensor* t, int64_t items, int64_t carry_elem
         k_merge_partition<uint64_t><<<blocks, 256, 0, stream>>>(static_cast<const uint64_t*>(t->pos[last]), nseg, nnz,
                                                                  items, p.nchunks, p.row, p.nz);
     SP_LAUNCH_CHECK();
+    sp_count_launches(1);
     t->parts[key] = p;
     *out = p;
     return SP_OK;
@@ -110,6 +111,7 @@ sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t per, cudaStream_t stream
             static_cast<const uint64_t*>(t->pos[1]), nslice, static_cast<const uint64_t*>(t->pos[2]), nfiber, nnz, per,
             p.nchunks, p.row, p.nz, p.aux);
     SP_LAUNCH_CHECK();
+    sp_count_launches(1);
     t->parts[key] = p;
     *out = p;
     return SP_OK;

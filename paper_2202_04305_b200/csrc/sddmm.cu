@@ -174,5 +174,6 @@ extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const 
     });
 #undef SP_SDDMM_LAUNCH
     SP_LAUNCH_CHECK();
+    sp_count_launches(2);
     return SP_OK;
 }

@@ -289,9 +289,11 @@ extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* str
             k_spmv<P, I, false><<<(unsigned)part.nchunks, kVThreads, 0, stream>>>(pos, crd, A->val, outer, x, y, part.row,
                                                                                   part.nz, nseg, cval, crow);
             k_spmv_fixup<I><<<(unsigned)sp_ceil_div(part.nchunks, 256), 256, 0, stream>>>(cval, crow, part.nchunks, outer, y);
+            sp_count_launches(2);
         } else {
             k_spmv<P, I, true><<<(unsigned)part.nchunks, kVThreads, 0, stream>>>(pos, crd, A->val, outer, x, y, part.row,
                                                                                  part.nz, nseg, cval, crow);
+            sp_count_launches(1);
         }
     });
     SP_LAUNCH_CHECK();
@@ -332,8 +334,10 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
         if (rowmajor) {
             if (vec2) SP_SPMM_LAUNCH(2, false); else SP_SPMM_LAUNCH(1, false);
             k_spmm_fixup<I><<<blocks, kMThreads, 0, stream>>>(carry, crow, part.nchunks, outer, N, C, ldc);
+            sp_count_launches(2);
         } else {
             if (vec2) SP_SPMM_LAUNCH(2, true); else SP_SPMM_LAUNCH(1, true);
+            sp_count_launches(1);
         }
     });
 #undef SP_SPMM_LAUNCH
