@@ -55,7 +55,8 @@ typedef enum {
     SP_ERR_DUPLICATE = 5,       /* SP_DUP_ERROR was set and two entries share coordinates */
     SP_ERR_ALLOC = 6,           /* the allocator returned NULL */
     SP_ERR_CUDA = 7,            /* a CUDA runtime call failed */
-    SP_ERR_TIMEOUT = 8          /* a bounded device-side wait ran out */
+    SP_ERR_TIMEOUT = 8,         /* a bounded device-side wait ran out */
+    SP_ERR_TOO_LARGE = 9        /* the problem does not fit a fixed-capacity entry point (sp_spmv_static) */
 } sp_status;
 
 /* flags of sp_pack */
@@ -166,6 +167,40 @@ sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const double* B, 
  */
 sp_status sp_mttkrp(sp_tensor* T, const double* B, const double* C, int64_t R,
                     double* M, void* stream);
+
+/*
+ * sp_spmv_static - y = A * x exactly as sp_spmv computes it (same encodings, same
+ * kernels, same results), for callers that are not allowed to allocate device memory.
+ * The paper has no counterpart; this is a deployment variant of sp_spmv.
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a real-time or
+ * safety-qualified loop whose memory must all be reserved at start-up, a plug-in
+ * living inside a host application that owns the GPU heap and forbids foreign
+ * allocations, or a service whose allocator may block or fail under memory
+ * pressure at exactly the moment the product is needed.  sp_spmv obtains its
+ * work-partition table and row-carry buffer through the allocator on a handle's
+ * first use; this call never does.  It calls neither the installed allocator nor
+ * cudaMalloc / cudaFree, and caches nothing in the handle.
+ *
+ * Its scratch is a fixed array compiled into the library (about 2 MiB of device
+ * memory on every GPU that loads the library, held until the process exits).
+ * Capacity: rows-or-columns stored at the compressed level plus stored entries,
+ * i.e. (sp_positions(A, 1) len - 1) + (sp_coordinates(A, 1) len), must not exceed
+ * SP_SPMV_STATIC_MAX_ITEMS; larger inputs are refused with SP_ERR_TOO_LARGE and
+ * nothing is launched.
+ *
+ * The first call on each device looks up the array's device address (a CUDA
+ * runtime query, no allocation); make that first call during set-up, before any
+ * stream capture is begun.  All calls share the one array: two calls whose
+ * kernels may overlap on the GPU (different streams, or different host threads
+ * on one device) race on it and give wrong results - serialise them.  The array
+ * keeps whatever the last call left; every word a call reads it has written
+ * itself earlier in that call, so no clearing is needed between calls.
+ * The partition is recomputed on every call (one small extra kernel).
+ * x, y, stream, errors and the atomics remark are as for sp_spmv; A is not modified.
+ */
+#define SP_SPMV_STATIC_MAX_ITEMS 134217728   /* 65,536 tiles of 2,048 (row end + entry) items */
+sp_status sp_spmv_static(const sp_tensor* A, const double* x, double* y, void* stream);
 
 /*
  * Measurement aids (no counterpart in the paper).

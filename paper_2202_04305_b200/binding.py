@@ -19,7 +19,8 @@ _LIB_PATH = os.path.join(_HERE, "libsp.so")
 
 SYMBOLS = ["sp_status_string", "sp_set_allocator", "sp_pack", "sp_free", "sp_info", "sp_positions",
            "sp_coordinates", "sp_values", "sp_unpack", "sp_spmv", "sp_spmm", "sp_sddmm", "sp_mttkrp",
-           "sp_set_profiling", "sp_get_pack_profile", "sp_launch_count"]
+           "sp_set_profiling", "sp_get_pack_profile", "sp_launch_count", "sp_spmv_static"]
+SPMV_STATIC_MAX_ITEMS = 134217728
 
 
 class SpError(RuntimeError):
@@ -197,6 +198,16 @@ def sp_spmv(A: SpTensor, x, y=None):
     if y is None:
         y = torch.empty(A.dims[0], dtype=torch.float64, device="cuda")
     _check(_lib.sp_spmv(A._h, _dptr(x), _dptr(y), _stream()), "sp_spmv")
+    return y
+
+
+def sp_spmv_static(A: SpTensor, x, y):
+    """sp_spmv for callers that may not allocate: the library's scratch is a fixed device array.
+
+    y must be supplied (this wrapper allocates nothing either).  Calls share that one array, so
+    do not let two of them overlap on the GPU; see include/sp.h for the capacity and the rules."""
+    _f64(x, "x"); _f64(y, "y")
+    _check(_lib.sp_spmv_static(A._h, _dptr(x), _dptr(y), _stream()), "sp_spmv_static")
     return y
 
 

@@ -40,6 +40,7 @@ const char* sp_status_string(sp_status s) {
         case SP_ERR_ALLOC: return "device allocation failed";
         case SP_ERR_CUDA: return "CUDA runtime error";
         case SP_ERR_TIMEOUT: return "bounded device-side wait ran out";
+        case SP_ERR_TOO_LARGE: return "problem exceeds the fixed scratch capacity of this entry point";
     }
     return "unknown status";
 }

@@ -344,3 +344,101 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
     SP_LAUNCH_CHECK();
     return SP_OK;
 }
+
+// ------------------------------------------------------------------ sp_spmv_static
+// SpMV whose scratch (merge-path partition table and row carries) is a fixed device array
+// compiled into the library instead of memory obtained at run time.
+namespace {
+
+constexpr int64_t kStaticMaxTiles = SP_SPMV_STATIC_MAX_ITEMS / kVTile;
+
+struct SpmvStaticScratch {
+    int64_t row[kStaticMaxTiles + 1];
+    int64_t nz[kStaticMaxTiles + 1];
+    double carry_val[kStaticMaxTiles];
+    int64_t carry_row[kStaticMaxTiles];
+};
+
+// About 2 MiB, resident on every GPU that loads the library until the process exits.
+static __device__ __align__(256) unsigned char g_spmv_static_scratch[sizeof(SpmvStaticScratch)];
+
+// In host code the symbol above is only a handle; the device address has to be asked for,
+// once per device, with that device current.
+std::mutex g_static_mu;
+void* g_static_addr[64] = {nullptr};
+
+sp_status spmv_static_scratch(SpmvStaticScratch** out) {
+    int dev = 0;
+    SP_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return SP_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_addr[dev]) {
+        void* p = nullptr;
+        SP_CUDA(cudaGetSymbolAddress(&p, g_spmv_static_scratch));
+        g_static_addr[dev] = p;
+    }
+    *out = static_cast<SpmvStaticScratch*>(g_static_addr[dev]);
+    return SP_OK;
+}
+
+// Same merge-path split as the cached partition tables, written into the fixed scratch.
+template <typename P>
+__global__ void k_static_partition(const P* __restrict__ pos, int64_t nseg, int64_t nnz, int64_t ntiles,
+                                   int64_t* __restrict__ row, int64_t* __restrict__ nz) {
+    const int64_t w = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (w > ntiles) return;
+    const int64_t total = nseg + nnz;
+    int64_t d = w * kVTile;
+    if (d > total) d = total;
+    int64_t lo = d > nnz ? d - nnz : 0;
+    int64_t hi = d < nseg ? d : nseg;
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if ((int64_t)pos[mid + 1] <= d - mid - 1) lo = mid + 1; else hi = mid;
+    }
+    row[w] = lo;
+    nz[w] = d - lo;
+}
+
+}  // namespace
+
+extern "C" sp_status sp_spmv_static(const sp_tensor* A, const double* x, double* y, void* stream_) {
+    if (!A || !x || !y) return SP_ERR_INVALID_ARG;
+    if (!matrix_encoding_ok(A)) return SP_ERR_UNSUPPORTED;
+    const int64_t nseg = A->npos[1] - 1;
+    const int64_t nnz = A->ncrd[1];
+    if (nseg + nnz > (int64_t)SP_SPMV_STATIC_MAX_ITEMS) return SP_ERR_TOO_LARGE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    SpmvStaticScratch* sc = nullptr;
+    sp_status st = spmv_static_scratch(&sc);
+    if (st != SP_OK) return st;
+    const bool rowmajor = A->ord[0] == 0;
+    const bool dbl = A->lt[0] == SP_COMPRESSED;
+    if (!rowmajor || dbl) SP_CUDA(cudaMemsetAsync(y, 0, (size_t)A->dims[0] * sizeof(double), stream));
+    if (nseg <= 0) return SP_OK;
+    int64_t ntiles = sp_ceil_div(nseg + nnz, kVTile);
+    if (ntiles < 1) ntiles = 1;
+    // Every scratch word read below is written earlier in this same call (the partition kernel
+    // fills row/nz for all tiles, each SpMV block writes its own carry slot), so nothing left by
+    // an earlier call is ever consumed and no clearing pass is needed.
+    SP_DISPATCH_WIDTHS(A, {
+        const P* pos = static_cast<const P*>(A->pos[1]);
+        const I* crd = static_cast<const I*>(A->crd[1]);
+        const I* outer = dbl ? static_cast<const I*>(A->crd[0]) : nullptr;
+        k_static_partition<P><<<(unsigned)sp_ceil_div(ntiles + 1, 256), 256, 0, stream>>>(pos, nseg, nnz, ntiles, sc->row,
+                                                                                          sc->nz);
+        if (rowmajor) {
+            k_spmv<P, I, false><<<(unsigned)ntiles, kVThreads, 0, stream>>>(pos, crd, A->val, outer, x, y, sc->row, sc->nz,
+                                                                            nseg, sc->carry_val, sc->carry_row);
+            k_spmv_fixup<I><<<(unsigned)sp_ceil_div(ntiles, 256), 256, 0, stream>>>(sc->carry_val, sc->carry_row, ntiles,
+                                                                                    outer, y);
+            sp_count_launches(3);
+        } else {
+            k_spmv<P, I, true><<<(unsigned)ntiles, kVThreads, 0, stream>>>(pos, crd, A->val, outer, x, y, sc->row, sc->nz,
+                                                                           nseg, sc->carry_val, sc->carry_row);
+            sp_count_launches(2);
+        }
+    });
+    SP_LAUNCH_CHECK();
+    return SP_OK;
+}
