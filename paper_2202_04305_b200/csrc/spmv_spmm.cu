@@ -26,9 +26,11 @@ k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __res
        const I* __restrict__ outer, const double* __restrict__ x, double* __restrict__ y,
        const int64_t* __restrict__ prow, const int64_t* __restrict__ pnz, int64_t nseg,
        double* __restrict__ carry_val, int64_t* __restrict__ carry_row) {
+    // a thread walks kVIpt consecutive products; one pad slot per kVIpt keeps those walks on distinct banks
     __shared__ int s_end[kVTile + 1];
-    __shared__ double s_prod[kVTile];
-    __shared__ I s_dst[SCATTER ? kVTile : 1];
+    __shared__ double s_prod[kVTile + kVTile / kVIpt];
+    __shared__ I s_dst[SCATTER ? kVTile + kVTile / kVIpt : 1];
+#define SP_PAD(i) ((i) + ((i) / kVIpt))
     __shared__ double s_wv[kVThreads / 32];
     __shared__ int s_wf[kVThreads / 32];
 
@@ -37,12 +39,53 @@ k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __res
     const int64_t i1 = prow[blockIdx.x + 1], j1 = pnz[blockIdx.x + 1];
     const int nrows = (int)(i1 - i0), nnzs = (int)(j1 - j0);
 
+    // All loads of the tile are issued before anything consumes them: kVIpt coordinates and values
+    // per thread, then the kVIpt gathered x entries (out-of-range slots re-read entry 0 and are dropped).
+    I cc[kVIpt];
+    double vv[kVIpt], xx[kVIpt];
+    if (nnzs > 0) {
+#pragma unroll
+        for (int it = 0; it < kVIpt; ++it) {
+            const int jj = t + it * kVThreads;
+            const int64_t g = j0 + (jj < nnzs ? jj : 0);
+            cc[it] = crd[g];
+            vv[it] = val[g];
+        }
+        if (!SCATTER) {
+#pragma unroll
+            for (int it = 0; it < kVIpt; ++it) xx[it] = __ldg(x + cc[it]);
+        }
+    }
+    if (!SCATTER && nrows == 0) {
+        // The whole tile lies inside one long row: no row ends to merge with, so the tile is a
+        // plain dot product - registers and one block reduction, no staging.
+        double s = 0.0;
+#pragma unroll
+        for (int it = 0; it < kVIpt; ++it)
+            if (t + it * kVThreads < nnzs) s = fma(vv[it], xx[it], s);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if ((t & 31) == 0) s_wv[t >> 5] = s;
+        __syncthreads();
+        if (t == 0) {
+            double tot = s_wv[0];
+#pragma unroll
+            for (int i = 1; i < kVThreads / 32; ++i) tot += s_wv[i];
+            carry_val[blockIdx.x] = tot;
+            carry_row[blockIdx.x] = (i1 < nseg && j1 > j0) ? i1 : -1;
+        }
+        return;
+    }
     for (int r = t; r < nrows; r += kVThreads) s_end[r] = (int)((int64_t)pos[i0 + r + 1] - j0);
-    for (int jj = t; jj < nnzs; jj += kVThreads) {
-        const I c = crd[j0 + jj];
-        const double v = val[j0 + jj];
-        if (SCATTER) { s_prod[jj] = v; s_dst[jj] = c; }
-        else s_prod[jj] = v * __ldg(x + c);
+    if (nnzs > 0) {
+#pragma unroll
+        for (int it = 0; it < kVIpt; ++it) {
+            const int jj = t + it * kVThreads;
+            if (jj < nnzs) {
+                if (SCATTER) { s_prod[SP_PAD(jj)] = vv[it]; s_dst[SP_PAD(jj)] = cc[it]; }
+                else s_prod[SP_PAD(jj)] = vv[it] * xx[it];
+            }
+        }
     }
     __syncthreads();
 
@@ -64,7 +107,7 @@ k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __res
                 ++ti; ++seg;
                 xc = seg < nseg ? x[outer ? (int64_t)outer[seg] : seg] : 0.0;
             } else {
-                atomicAdd(y + (int64_t)s_dst[tj], s_prod[tj] * xc);
+                atomicAdd(y + (int64_t)s_dst[SP_PAD(tj)], s_prod[SP_PAD(tj)] * xc);
                 ++tj;
             }
         }
@@ -83,7 +126,7 @@ k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __res
             run = 0.0;
             ++ti;
         } else {
-            run += s_prod[tj];
+            run += s_prod[SP_PAD(tj)];
             ++tj;
         }
     }
@@ -118,6 +161,7 @@ k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __res
         carry_val[blockIdx.x] = outv;
         carry_row[blockIdx.x] = (i1 < nseg && j1 > j0) ? i1 : -1;
     }
+#undef SP_PAD
 }
 
 template <typename I>
