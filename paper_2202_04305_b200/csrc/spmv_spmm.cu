@@ -13,6 +13,8 @@
 // Column-major encodings scatter into the output with f64 atomic adds.
 #include "common.cuh"
 
+#include <limits.h>
+
 namespace {
 
 // ===================================================================== SpMV
@@ -284,6 +286,106 @@ k_spmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __res
     if (!SCATTER && lane == 0) carry_row[w] = (j1 > pstart && i1 < nseg) ? i1 : -1;
 }
 
+// Row-major SpMM (CSR, DCSR).  A warp walks its merge-path piece 32 entries at a time; lane = output
+// column(s).  The ends of the rows that fall inside a batch come from a 32-row window of pos[] as a
+// bit mask, so the loads of the batch do not depend on the row structure: B rows are fetched in
+// groups of kGather independent loads, then accumulated in order, and a row is stored when its end
+// bit comes up (rows without entries that end at the same place are stored as zeros).
+constexpr int kGather = 8;
+
+template <typename P, typename I, int V>
+__global__ void __launch_bounds__(kMThreads)
+k_spmm_gather(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
+              const I* __restrict__ outer, const double* __restrict__ B, int64_t N, int64_t ldb,
+              double* __restrict__ C, int64_t ldc, const int64_t* __restrict__ prow,
+              const int64_t* __restrict__ pnz, int64_t nchunks, int64_t nseg, double* __restrict__ carry,
+              int64_t* __restrict__ carry_row) {
+    const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    if (w >= nchunks) return;
+    const int lane = threadIdx.x & 31;
+    const int64_t i0 = prow[w], j0 = pnz[w], i1 = prow[w + 1], j1 = pnz[w + 1];
+    constexpr int64_t kInf = INT64_MAX;
+    int64_t pstart = j0;
+
+    for (int64_t cbase = 0; cbase < N; cbase += 32 * V) {
+        const int64_t col = cbase + (int64_t)lane * V;
+        const bool on = col < N;
+        const double* Bc = B + (on ? col : cbase);        // idle lanes read a valid column and never write
+        double acc[V];
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc[q] = 0.0;
+        int64_t row = i0, p = j0, rbase = i0;
+        pstart = j0;
+        int64_t E = (rbase + lane < i1) ? (int64_t)pos[rbase + lane + 1] : kInf;
+        I c_n = (p + lane < j1) ? crd[p + lane] : (I)0;
+        double v_n = (p + lane < j1) ? val[p + lane] : 0.0;
+
+        // stores `acc` as row `row`, then zero rows for the other rows of the window that end at `pe`
+        auto close_rows = [&](int64_t pe) {
+            const int same = __popc(__ballot_sync(0xffffffffu, E == pe));
+            for (int r = 0; r < same; ++r) {
+                if (on) st_vec<V>(C + (outer ? (int64_t)outer[row] : row) * ldc + col, acc);
+#pragma unroll
+                for (int q = 0; q < V; ++q) acc[q] = 0.0;
+                ++row;
+            }
+            pstart = pe;
+        };
+
+        // every turn of this loop either closes at least one row or consumes at least one entry;
+        // `budget` bounds the turns all the same, so a malformed pos[] cannot spin a warp for ever
+        for (int64_t budget = (i1 - i0) + (j1 - j0) + 2; budget > 0; --budget) {
+            if (row - rbase >= 32) {              // the window is used up (also when row == i1)
+                rbase += 32;
+                E = (rbase + lane < i1) ? (int64_t)pos[rbase + lane + 1] : kInf;
+            }
+            // rows that end exactly here: the open row if it is complete, and rows without entries
+            if (row < i1 && __shfl_sync(0xffffffffu, E, (int)(row - rbase)) == p) {
+                close_rows(p);
+                continue;
+            }
+            if (p >= j1) break;
+            const int64_t elast = __shfl_sync(0xffffffffu, E, 31);
+            int64_t lim = j1 - p;
+            if (elast - p < lim) lim = elast - p;
+            const int cnt = lim < 32 ? (int)lim : 32;
+            if (cnt <= 0) break;                  // cannot happen for a well-formed pos[]
+            const I c_l = c_n;
+            const double v_l = v_n;
+            {
+                const int64_t pn = p + cnt;
+                c_n = (pn + lane < j1) ? crd[pn + lane] : (I)0;
+                v_n = (pn + lane < j1) ? val[pn + lane] : 0.0;
+            }
+            const int64_t rel = E - p - 1;
+            const unsigned endmask = __reduce_or_sync(0xffffffffu, (rel >= 0 && rel < cnt) ? (1u << (int)rel) : 0u);
+
+            for (int g = 0; g < cnt; g += kGather) {
+                vec_t<V> b[kGather];
+#pragma unroll
+                for (int u = 0; u < kGather; ++u) {
+                    if (g + u < cnt) {
+                        const int64_t k = (int64_t)__shfl_sync(0xffffffffu, c_l, g + u);
+                        b[u] = ld_vec<V>(Bc + k * ldb);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kGather; ++u) {
+                    if (g + u < cnt) {
+                        const double vv = __shfl_sync(0xffffffffu, v_l, g + u);
+#pragma unroll
+                        for (int q = 0; q < V; ++q) acc[q] = fma(vv, b[u].a[q], acc[q]);
+                        if ((endmask >> (g + u)) & 1u) close_rows(p + g + u + 1);
+                    }
+                }
+            }
+            p += cnt;
+        }
+        if (on && j1 > pstart) st_vec<V>(carry + w * N + col, acc);
+    }
+    if (lane == 0) carry_row[w] = (j1 > pstart && i1 < nseg) ? i1 : -1;
+}
+
 template <typename I>
 __global__ void k_spmm_fixup(const double* __restrict__ carry, const int64_t* __restrict__ carry_row,
                              int64_t nchunks, const I* __restrict__ outer, int64_t N, double* __restrict__ C,
@@ -376,7 +478,12 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
         const I* crd = static_cast<const I*>(A->crd[1]);
         const I* outer = dbl ? static_cast<const I*>(A->crd[0]) : nullptr;
         if (rowmajor) {
-            if (vec2) SP_SPMM_LAUNCH(2, false); else SP_SPMM_LAUNCH(1, false);
+            if (vec2)
+                k_spmm_gather<P, I, 2><<<blocks, kMThreads, 0, stream>>>(pos, crd, A->val, outer, B, N, ldb, C, ldc, part.row,
+                                                                         part.nz, part.nchunks, nseg, carry, crow);
+            else
+                k_spmm_gather<P, I, 1><<<blocks, kMThreads, 0, stream>>>(pos, crd, A->val, outer, B, N, ldb, C, ldc, part.row,
+                                                                         part.nz, part.nchunks, nseg, carry, crow);
             k_spmm_fixup<I><<<blocks, kMThreads, 0, stream>>>(carry, crow, part.nchunks, outer, N, C, ldc);
             sp_count_launches(2);
         } else {
