@@ -46,7 +46,47 @@ __global__ void k_mttkrp_partition(const P* __restrict__ pos1, int64_t nslice, c
     nz[w] = p; fiber[w] = f; slice[w] = lo;
 }
 
+// One thread per stored entry: the segment (level-0 node) that holds it, by binary search in pos[1],
+// mapped through crd[0] when level 0 is compressed.
+template <typename P, typename I>
+__global__ void k_segment_ids(const P* __restrict__ pos, int64_t nseg, int64_t nnz, const I* __restrict__ outer,
+                              uint32_t* __restrict__ seg) {
+    const int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (p >= nnz) return;
+    int64_t lo = 0, hi = nseg;              // last q with pos[q] <= p  (pos[nseg] = nnz > p)
+    while (hi - lo > 1) {
+        const int64_t mid = (lo + hi) >> 1;
+        if ((int64_t)pos[mid] <= p) lo = mid; else hi = mid;
+    }
+    seg[p] = outer ? (uint32_t)outer[lo] : (uint32_t)lo;
+}
+
 }  // namespace
+
+sp_status sp_get_segment_ids(sp_tensor* t, cudaStream_t stream, const uint32_t** out) {
+    std::lock_guard<std::mutex> lock(t->mu);
+    const uint64_t key = (uint64_t)SP_PART_SEGIDS << 56;
+    auto it = t->parts.find(key);
+    if (it != t->parts.end()) { *out = reinterpret_cast<const uint32_t*>(it->second.aux); return SP_OK; }
+    const int64_t nseg = t->npos[1] - 1, nnz = t->ncrd[1];
+    sp_partition p;
+    p.aux = static_cast<int64_t*>(sp_dev_alloc((size_t)(nnz ? nnz : 1) * sizeof(uint32_t), stream));
+    if (!p.aux) return SP_ERR_ALLOC;
+    uint32_t* seg = reinterpret_cast<uint32_t*>(p.aux);
+    if (nnz > 0) {
+        const unsigned blocks = (unsigned)sp_ceil_div(nnz, 256);
+        SP_DISPATCH_WIDTHS(t, {
+            k_segment_ids<P, I><<<blocks, 256, 0, stream>>>(static_cast<const P*>(t->pos[1]), nseg, nnz,
+                                                           t->lt[0] == SP_COMPRESSED ? static_cast<const I*>(t->crd[0]) : nullptr,
+                                                           seg);
+        });
+        SP_LAUNCH_CHECK();
+        sp_count_launches(1);
+    }
+    t->parts[key] = p;
+    *out = seg;
+    return SP_OK;
+}
 
 sp_status sp_get_merge_partition(sp_tensor* t, int64_t items, int64_t carry_elems_per_chunk, cudaStream_t stream,
                                  sp_partition* out) {

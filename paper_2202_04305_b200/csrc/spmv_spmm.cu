@@ -305,6 +305,7 @@ k_spmm_gather(const P* __restrict__ pos, const I* __restrict__ crd, const double
     const int lane = threadIdx.x & 31;
     const int64_t i0 = prow[w], j0 = pnz[w], i1 = prow[w + 1], j1 = pnz[w + 1];
     constexpr int64_t kInf = INT64_MAX;
+    constexpr int kG = V == 2 ? kGather / 2 : kGather;   // same bytes in flight either way
     int64_t pstart = j0;
 
     for (int64_t cbase = 0; cbase < N; cbase += 32 * V) {
@@ -360,17 +361,17 @@ k_spmm_gather(const P* __restrict__ pos, const I* __restrict__ crd, const double
             const int64_t rel = E - p - 1;
             const unsigned endmask = __reduce_or_sync(0xffffffffu, (rel >= 0 && rel < cnt) ? (1u << (int)rel) : 0u);
 
-            for (int g = 0; g < cnt; g += kGather) {
-                vec_t<V> b[kGather];
+            for (int g = 0; g < cnt; g += kG) {
+                vec_t<V> b[kG];
 #pragma unroll
-                for (int u = 0; u < kGather; ++u) {
+                for (int u = 0; u < kG; ++u) {
                     if (g + u < cnt) {
                         const int64_t k = (int64_t)__shfl_sync(0xffffffffu, c_l, g + u);
                         b[u] = ld_vec<V>(Bc + k * ldb);
                     }
                 }
 #pragma unroll
-                for (int u = 0; u < kGather; ++u) {
+                for (int u = 0; u < kG; ++u) {
                     if (g + u < cnt) {
                         const double vv = __shfl_sync(0xffffffffu, v_l, g + u);
 #pragma unroll
@@ -384,6 +385,58 @@ k_spmm_gather(const P* __restrict__ pos, const I* __restrict__ crd, const double
         if (on && j1 > pstart) st_vec<V>(carry + w * N + col, acc);
     }
     if (lane == 0) carry_row[w] = (j1 > pstart && i1 < nseg) ? i1 : -1;
+}
+
+// Column-major SpMM (CSC, DCSC): C[i,:] += A[i,k] * B[k,:] for every stored entry, as a flat loop
+// over entries.  seg[p] is the column k of entry p (expanded once per handle), crd[p] its row i.
+// A warp takes kScatPer consecutive entries, 32 at a time; lane = output column.  Entries of one
+// column are adjacent, so the B row they share is read from DRAM once and then from L1; C is
+// updated with f64 atomic adds (it was zeroed by the caller).
+constexpr int kScatPer = 256;
+
+template <typename I, int V>
+__global__ void __launch_bounds__(kMThreads)
+k_spmm_scatter(const uint32_t* __restrict__ seg, const I* __restrict__ crd, const double* __restrict__ val,
+               int64_t nnz, const double* __restrict__ B, int64_t N, int64_t ldb, double* __restrict__ C,
+               int64_t ldc) {
+    const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    const int64_t p0 = w * kScatPer;
+    if (p0 >= nnz) return;
+    const int64_t p1 = p0 + kScatPer < nnz ? p0 + kScatPer : nnz;
+    for (int64_t cbase = 0; cbase < N; cbase += 32 * V) {
+        const int64_t col = cbase + (int64_t)lane * V;
+        const bool on = col < N;
+        const double* Bc = B + (on ? col : cbase);
+        double* Cc = C + (on ? col : cbase);
+        for (int64_t p = p0; p < p1; p += 32) {
+            const int cnt = p1 - p < 32 ? (int)(p1 - p) : 32;
+            const uint32_t k_l = lane < cnt ? seg[p + lane] : 0u;
+            const I i_l = lane < cnt ? crd[p + lane] : (I)0;
+            const double v_l = lane < cnt ? val[p + lane] : 0.0;
+            for (int g = 0; g < cnt; g += kGather) {
+                vec_t<V> b[kGather];
+#pragma unroll
+                for (int u = 0; u < kGather; ++u) {
+                    if (g + u < cnt) {
+                        const int64_t k = (int64_t)__shfl_sync(0xffffffffu, k_l, g + u);
+                        b[u] = ld_vec<V>(Bc + k * ldb);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kGather; ++u) {
+                    if (g + u < cnt) {
+                        const int64_t i = (int64_t)__shfl_sync(0xffffffffu, i_l, g + u);
+                        const double vv = __shfl_sync(0xffffffffu, v_l, g + u);
+                        if (on) {
+#pragma unroll
+                            for (int q = 0; q < V; ++q) atomicAdd(Cc + i * ldc + q, vv * b[u].a[q]);
+                        }
+                    }
+                }
+            }
+        }
+    }
 }
 
 template <typename I>
@@ -461,9 +514,18 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
     }
     const int64_t nseg = A->npos[1] - 1;
     if (nseg <= 0) return SP_OK;
+    // column-major storage runs as a flat loop over entries with their column ids expanded once
+    const uint32_t* segs = nullptr;
+    sp_status st = SP_OK;
+    if (!rowmajor && A->dims[1] < ((int64_t)1 << 32)) {
+        st = sp_get_segment_ids(A, stream, &segs);
+        if (st != SP_OK) return st;
+    }
     sp_partition part;
-    sp_status st = sp_get_merge_partition(A, kMItems, N, stream, &part);
-    if (st != SP_OK) return st;
+    if (!segs) {
+        st = sp_get_merge_partition(A, kMItems, N, stream, &part);
+        if (st != SP_OK) return st;
+    }
     double* carry = part.carry;
     int64_t* crow = reinterpret_cast<int64_t*>(part.carry + part.nchunks * N);
     const bool vec2 = N > 32 && (N % 2 == 0) && (ldb % 2 == 0) && (ldc % 2 == 0) &&
@@ -486,6 +548,14 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
                                                                          part.nz, part.nchunks, nseg, carry, crow);
             k_spmm_fixup<I><<<blocks, kMThreads, 0, stream>>>(carry, crow, part.nchunks, outer, N, C, ldc);
             sp_count_launches(2);
+        } else if (segs) {
+            const int64_t nnz = A->ncrd[1];
+            const unsigned sblocks = (unsigned)sp_ceil_div(sp_ceil_div(nnz, kScatPer) * 32, kMThreads);
+            if (nnz > 0) {
+                if (vec2) k_spmm_scatter<I, 2><<<sblocks, kMThreads, 0, stream>>>(segs, crd, A->val, nnz, B, N, ldb, C, ldc);
+                else k_spmm_scatter<I, 1><<<sblocks, kMThreads, 0, stream>>>(segs, crd, A->val, nnz, B, N, ldb, C, ldc);
+                sp_count_launches(1);
+            }
         } else {
             if (vec2) SP_SPMM_LAUNCH(2, true); else SP_SPMM_LAUNCH(1, true);
             sp_count_launches(1);
