@@ -183,7 +183,7 @@ class ClockSampler:
         self.p = None
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.Q}",
-                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                       "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.f,
                                       stderr=subprocess.DEVNULL)
         except Exception:
             pass
@@ -305,7 +305,7 @@ def run_reference(args, wl, model, total_flops, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--small", action="store_true", help="reduced sizes (development runs; not a valid benchmark)")
@@ -345,14 +345,14 @@ def main():
     suite = GpuSuite(wl)
 
     # ---- whole-step throughput, inputs resident in HBM
-    for _ in range(args.warmup):
-        suite.step()
-    torch.cuda.synchronize(); dist_barrier()
     try:
         gpu_id = "GPU-" + str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
     except Exception:
         gpu_id = str(local_rank)
-    sampler = ClockSampler(gpu_id)
+    sampler = ClockSampler(gpu_id)          # samples through warm-up and the timed steps (all under load)
+    for _ in range(args.warmup):
+        suite.step()
+    torch.cuda.synchronize(); dist_barrier()
     l0 = sp.sp_launch_count()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if args.only_step:

@@ -127,21 +127,41 @@ __device__ __forceinline__ uint32_t block256_excl_scan(uint32_t v, uint32_t* sum
 __global__ void __launch_bounds__(kSortThreads)
 k_sort_upsweep(const uint64_t* __restrict__ keys, int64_t n, int shift, uint32_t mask,
                uint32_t* __restrict__ tilehist, int64_t ntiles) {
-    __shared__ uint32_t hist[kRadix];
-    const int t = threadIdx.x;
-    hist[t] = 0;
+    __shared__ uint32_t hist[kSortWarps][kRadix];     // one histogram per warp: conflicts only inside a warp
+    const int t = threadIdx.x, w = t >> 5;
+#pragma unroll
+    for (int i = 0; i < kSortWarps; ++i) hist[i][t] = 0;
     __syncthreads();
     const int64_t base = (int64_t)blockIdx.x * kSortTile;
-#pragma unroll 4
+    uint64_t k[kSortIpt];
+#pragma unroll
+    for (int i = 0; i < kSortIpt; ++i) {             // all loads first
+        const int64_t e = base + (int64_t)i * kSortThreads + t;
+        k[i] = e < n ? keys[e] : 0;
+    }
+#pragma unroll
     for (int i = 0; i < kSortIpt; ++i) {
-        int64_t e = base + (int64_t)i * kSortThreads + t;
-        bool valid = e < n;
-        uint32_t d = valid ? ((uint32_t)(keys[e] >> shift) & mask) : (uint32_t)kRadix;
-        uint32_t peers = __match_any_sync(0xffffffffu, d);
-        if (valid && (int)sp_lane() == __ffs(peers) - 1) atomicAdd(&hist[d], (uint32_t)__popc(peers));
+        const int64_t e = base + (int64_t)i * kSortThreads + t;
+        if (e < n) atomicAdd(&hist[w][(uint32_t)(k[i] >> shift) & mask], 1u);
     }
     __syncthreads();
-    tilehist[(int64_t)t * ntiles + blockIdx.x] = hist[t];
+    uint32_t c = 0;
+#pragma unroll
+    for (int i = 0; i < kSortWarps; ++i) c += hist[i][t];
+    tilehist[(int64_t)t * ntiles + blockIdx.x] = c;
+}
+
+// Lanes of the warp whose 9-bit value (digit, or kRadix for padding) equals this lane's, by one
+// ballot per bit.  (A hardware match instruction does the same but costs far more per call.)
+__device__ __forceinline__ uint32_t same_value_lanes(uint32_t d) {
+    uint32_t peers = 0xffffffffu;
+#pragma unroll
+    for (int b = 0; b < 9; ++b) {
+        const bool bit = (d >> b) & 1u;
+        const uint32_t bal = __ballot_sync(0xffffffffu, bit);
+        peers &= bit ? bal : ~bal;
+    }
+    return peers;
 }
 
 // One block per digit: exclusive scan of that digit's tile counts, in place.
@@ -164,7 +184,7 @@ k_sort_scan(uint32_t* tilehist, int64_t ntiles, uint32_t* digit_total) {
 constexpr size_t kDownSmem = (size_t)kSortTile * 8 + (size_t)kSortTile * 4 +
                              (size_t)kSortWarps * (kRadix + 1) * 4 + (size_t)(kRadix + 1) * 4 + (size_t)kRadix * 8 + 64;
 
-__global__ void __launch_bounds__(kSortThreads)
+__global__ void __launch_bounds__(kSortThreads, 3)   // three tiles per SM hide the ranking chain's latency
 k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict__ idx_in,
                  uint64_t* __restrict__ keys_out, uint32_t* __restrict__ idx_out, int64_t n, int shift,
                  uint32_t mask, const uint32_t* __restrict__ tilehist, int64_t ntiles,
@@ -190,19 +210,23 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
     uint32_t* mycnt = wcnt + w * (kRadix + 1);
     const uint32_t lt_mask = (1u << lane) - 1u;
 #pragma unroll
-    for (int i = 0; i < kSortIpt; ++i) {
-        int li = w * (32 * kSortIpt) + i * 32 + lane;
-        bool valid = li < tile_n;
+    for (int i = 0; i < kSortIpt; ++i) {             // all loads first
+        const int li = w * (32 * kSortIpt) + i * 32 + lane;
+        const bool valid = li < tile_n;
         key[i] = valid ? keys_in[base + li] : 0;
         pay[i] = valid ? idx_in[base + li] : 0;
-        uint32_t d = valid ? ((uint32_t)(key[i] >> shift) & mask) : (uint32_t)kRadix;
-        uint32_t peers = __match_any_sync(0xffffffffu, d);
-        int leader = __ffs(peers) - 1;
+    }
+#pragma unroll
+    for (int i = 0; i < kSortIpt; ++i) {
+        const int li = w * (32 * kSortIpt) + i * 32 + lane;
+        const uint32_t d = li < tile_n ? ((uint32_t)(key[i] >> shift) & mask) : (uint32_t)kRadix;
+        const uint32_t peers = __match_any_sync(0xffffffffu, d);
+        const int leader = __ffs(peers) - 1;
         uint32_t b = 0;
         if (lane == leader) { b = mycnt[d]; mycnt[d] = b + (uint32_t)__popc(peers); }
         b = __shfl_sync(0xffffffffu, b, leader);
         rank[i] = b + (uint32_t)__popc(peers & lt_mask);
-        __syncwarp();
+        __syncwarp();                                 // rounds update the same counters: keep them in order
     }
     __syncthreads();
 
@@ -380,6 +404,15 @@ __global__ void __launch_bounds__(kCtThreads) k_emit(EmitArgs a) {
     for (int l = 0; l < SP_MAX_RANK; ++l)
         incl[l] = a.tileprefix[(int64_t)l * a.ntiles + blockIdx.x] + (int64_t)((ex >> (kField * l)) & kFieldMask);
 
+    // values of this thread's entries, gathered before the (sequential) level walk needs them
+    uint32_t id[kCtIpt];
+    double vin[kCtIpt];
+#pragma unroll
+    for (int i = 0; i < kCtIpt; ++i) id[i] = (e0 + i < a.n) ? a.idx[e0 + i] : 0u;
+#pragma unroll
+    for (int i = 0; i < kCtIpt; ++i) vin[i] = a.vals_in[(e0 + i < a.n) ? id[i] : 0u];
+    const bool next_same = (e0 + kCtIpt < a.n) && a.keys[e0 + kCtIpt] == k[kCtIpt - 1];
+
     uint64_t kp = kprev;
 #pragma unroll
     for (int i = 0; i < kCtIpt; ++i) {
@@ -410,8 +443,12 @@ __global__ void __launch_bounds__(kCtThreads) k_emit(EmitArgs a) {
             }
         }
         if (full) {
-            double s = a.vals_in[a.idx[e]];
-            for (int64_t g = e + 1; g < a.n && a.keys[g] == k[i]; ++g) s += a.vals_in[a.idx[g]];
+            // the entry after this one repeats the coordinates only when its "new position" flag is clear
+            const bool dup = (i + 1 < kCtIpt) ? (e + 1 < a.n && !((f[(i + 1) % kCtIpt] >> (kField * (p.rank - 1))) & 1))
+                                              : next_same;
+            double s = vin[i];
+            if (dup)
+                for (int64_t g = e + 1; g < a.n && a.keys[g] == k[i]; ++g) s += a.vals_in[a.idx[g]];
             a.val[ppos] = s;
         } else if (a.flags & SP_DUP_ERROR) {
             atomicOr(a.err, kErrDup);
