@@ -4,7 +4,7 @@
 A step is one pass of the whole path over the synthetic suite:
   pack(CSC) + pack(DCSR) + SpMM(CSC) + SpMM(DCSR) + SpMV(DCSR)   on the 1,048,576^2 / 5M-entry matrix (N = 32)
   SpMM(CSR, N = 64)                                               on the 65,536^2 power-law matrix
-  SpMV(CSR)                                                       on the 65,536^2 row band (first 1000 rows dense)
+  SpMV(CSR) + SpMV(CDR = compressed, dense)                       on the 65,536^2 row band (first 1000 rows dense)
   SDDMM(CSR, K = 128)                                             on the 131,072^2 / 2M-entry pattern
   pack(CSF) + MTTKRP(R = 32)                                      on the 16,384^3 / 20M-entry tensor
 `value` is the f64 GFLOP/s of the step (flops of the four compute kernels over the whole step
@@ -84,6 +84,9 @@ def work_model(wl):
     k["spmv_dcsr"] = dict(flops=2 * c3.nnz, bytes=12 * c3.nnz + 2 * W * rows3 + 8 * (n3 + m3))
     k["spmm_csr"] = dict(flops=2 * N2 * c2.nnz, bytes=12 * c2.nnz + W * (c2.dims[0] + 1) + 8 * N2 * sum(c2.dims))
     k["spmv_csr"] = dict(flops=2 * c1b.nnz, bytes=12 * c1b.nnz + W * (c1b.dims[0] + 1) + 8 * sum(c1b.dims))
+    dense_rows = int(np.unique(c1b.coords[0]).size) if "rows1b" not in wl else wl["rows1b"]
+    wl["rows1b"] = dense_rows
+    k["spmv_cdr"] = dict(flops=2 * dense_rows * c1b.dims[1], bytes=8 * dense_rows * c1b.dims[1] + 2 * W * dense_rows + 8 * sum(c1b.dims))
     k["sddmm_csr"] = dict(flops=c4.nnz * (2 * K4 + 1), bytes=20 * c4.nnz + W * (c4.dims[0] + 1) + 8 * K4 * sum(c4.dims))
     k["pack_csf"] = dict(flops=0, bytes=c5.nnz * 20 + c5.nnz * 12 + 2 * W * F5, units=c5.nnz)
     k["mttkrp_csf"] = dict(flops=2 * R5 * (c5.nnz + F5), bytes=12 * c5.nnz + 2 * W * F5 + 8 * R5 * sum(c5.dims))
@@ -108,6 +111,7 @@ class GpuSuite:
         self.M5 = f64(wl["c5"].dims[0], 32)
         self.A2 = sp.sp_pack(wl["c2"].dims, i32(wl["c2"]), dev(wl["c2"].vals), (0, 1))
         self.A1b = sp.sp_pack(wl["c1b"].dims, i32(wl["c1b"]), dev(wl["c1b"].vals), (0, 1))
+        self.A1c = sp.sp_pack(wl["c1b"].dims, i32(wl["c1b"]), dev(wl["c1b"].vals), (1, 0))
         self.S4 = sp.sp_pack(wl["c4"].dims, i32(wl["c4"]), dev(wl["c4"].vals), (0, 1))
         self.xv4 = f64(self.S4.nval)
         self.flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
@@ -123,6 +127,7 @@ class GpuSuite:
         sp.sp_spmv(a_dcsr, self.x3, self.y3)
         sp.sp_spmm(self.A2, self.B2, self.C2)
         sp.sp_spmv(self.A1b, self.x1b, self.y1b)
+        sp.sp_spmv(self.A1c, self.x1b, self.y1b)
         sp.sp_sddmm(self.S4, self.A4, self.B4, self.xv4)
         t5 = sp.sp_pack(wl["c5"].dims, self.c5, self.v5, (1, 1, 1))
         sp.sp_mttkrp(t5, self.Bf, self.Cf, self.M5)
@@ -151,6 +156,7 @@ class GpuSuite:
             "spmv_dcsr": lambda: sp.sp_spmv(dcsr(), self.x3, self.y3),
             "spmm_csr": lambda: sp.sp_spmm(self.A2, self.B2, self.C2),
             "spmv_csr": lambda: sp.sp_spmv(self.A1b, self.x1b, self.y1b),
+            "spmv_cdr": lambda: sp.sp_spmv(self.A1c, self.x1b, self.y1b),
             "sddmm_csr": lambda: sp.sp_sddmm(self.S4, self.A4, self.B4, self.xv4),
             "pack_csf": lambda: sp.sp_pack(wl["c5"].dims, self.c5, self.v5, (1, 1, 1)).free(),
             "mttkrp_csf": lambda: sp.sp_mttkrp(csf(), self.Bf, self.Cf, self.M5),
@@ -246,7 +252,7 @@ def oracle_sample(wl, small: bool):
     Returns (seconds spent, extrapolated seconds for a full step, description)."""
     import oracle as O
     O.lib()
-    frac = 1 if small else 10
+    frac = 1          # the whole lists, except where a line below says otherwise (about 20 s of CPU work)
     c3, c2, c1b, c4, c5 = wl["c3"], wl["c2"], wl["c1b"], wl["c4"], wl["c5"]
     spent = 0.0
     full = 0.0
@@ -269,6 +275,8 @@ def oracle_sample(wl, small: bool):
     run("spmm N=64 power-law matrix, all entries", lambda: O.spmm(c2.dims[0], c2.coords[0], c2.coords[1], c2.vals, wl["B2"]), 1)
     n1 = c1b.nnz // frac
     run("spmv row band 1/%d" % frac, lambda: O.spmv(c1b.dims[0], c1b.coords[0][:n1], c1b.coords[1][:n1], c1b.vals[:n1], wl["x1b"]), c1b.nnz / n1)
+    run("spmv row band again (the CDR call computes the same product)",
+        lambda: O.spmv(c1b.dims[0], c1b.coords[0][:n1], c1b.coords[1][:n1], c1b.vals[:n1], wl["x1b"]), c1b.nnz / n1)
     n4 = c4.nnz // frac
     run("sddmm 1/%d" % frac, lambda: O.sddmm(c4.coords[0][:n4], c4.coords[1][:n4], c4.vals[:n4], wl["A4"], wl["B4"]), c4.nnz / n4)
     n5 = c5.nnz // (2 * frac)
@@ -323,7 +331,7 @@ def main():
     total_bytes = sum(v["bytes"] for v in model.values())
     cfg = {"workload": ("SMALL development sizes" if args.small else
                         "suite: pack+SpMM+SpMV on 1,048,576^2/5M nnz (CSC, DCSR, N=32); SpMM CSR 65,536^2 power-law N=64; "
-                        "SpMV CSR 65,536^2 row band (65.5M nnz); SDDMM CSR 131,072^2/2M nnz K=128; "
+                        "SpMV CSR and CDR 65,536^2 row band (65.5M nnz); SDDMM CSR 131,072^2/2M nnz K=128; "
                         "pack+MTTKRP CSF 16,384^3/20M nnz R=32"),
            "index_bits": 32, "l2": "step inputs exceed L2 (about 3 GB touched per step); per-kernel timings flush L2 "
                                    "with a 512 MiB write between repetitions",
@@ -458,6 +466,7 @@ def run_e2e(suite, wl, args, total_flops, world):
             "y3": torch.empty(suite.y3.shape, dtype=torch.float64).pin_memory(),
             "C2": torch.empty(suite.C2.shape, dtype=torch.float64).pin_memory(),
             "y1b": torch.empty(suite.y1b.shape, dtype=torch.float64).pin_memory(),
+            "y1c": torch.empty(suite.y1b.shape, dtype=torch.float64).pin_memory(),
             "xv4": torch.empty(suite.xv4.shape, dtype=torch.float64).pin_memory(),
             "M5": torch.empty(suite.M5.shape, dtype=torch.float64).pin_memory()}
     h2d = sum(t.numel() * t.element_size() for k, v in h.items() for t in (v if isinstance(v, list) else [v]))
@@ -477,6 +486,7 @@ def run_e2e(suite, wl, args, total_flops, world):
         sp.sp_spmm(suite.A2, suite.B2, suite.C2); outs["C2"].copy_(suite.C2, non_blocking=True)
         suite.x1b.copy_(h["x1b"], non_blocking=True)
         sp.sp_spmv(suite.A1b, suite.x1b, suite.y1b); outs["y1b"].copy_(suite.y1b, non_blocking=True)
+        sp.sp_spmv(suite.A1c, suite.x1b, suite.y1b); outs["y1c"].copy_(suite.y1b, non_blocking=True)
         suite.A4.copy_(h["A4"], non_blocking=True); suite.B4.copy_(h["B4"], non_blocking=True)
         sp.sp_sddmm(suite.S4, suite.A4, suite.B4, suite.xv4); outs["xv4"].copy_(suite.xv4, non_blocking=True)
         for d, s in zip(suite.c5, h["c5"]):

@@ -131,8 +131,10 @@ sp_status sp_unpack(const sp_tensor* t, void* const* coo_coords_out, double* val
 
 /*
  * sp_spmv - y[i] = sum_k A[i,k] * x[k]  (the matvec of Section 6.2).
- * A: rank 2, level types (dense, compressed) or (compressed, compressed),
- * either ordering (CSR, DCSR, CSC, DCSC).  x has dims[1] entries, y dims[0].
+ * A: rank 2, any of the eight encodings: level types (dense, compressed) or
+ * (compressed, compressed) in either ordering (CSR, DCSR, CSC, DCSC), and
+ * (compressed, dense) - the "CDR" of Section 6.2 - or (dense, dense) in either
+ * ordering.  x has dims[1] entries, y dims[0].
  * Rows without stored entries are written as 0.  Column-major encodings
  * accumulate with floating-point atomics: the summation order, and so the
  * last bits, may differ from run to run.
@@ -169,8 +171,9 @@ sp_status sp_mttkrp(sp_tensor* T, const double* B, const double* C, int64_t R,
                     double* M, void* stream);
 
 /*
- * sp_spmv_static - y = A * x exactly as sp_spmv computes it (same encodings, same
- * kernels, same results), for callers that are not allowed to allocate device memory.
+ * sp_spmv_static - y = A * x exactly as sp_spmv computes it (same kernels, same
+ * results; the four encodings with a compressed inner level: CSR, DCSR, CSC, DCSC),
+ * for callers that are not allowed to allocate device memory.
  * The paper has no counterpart; this is a deployment variant of sp_spmv.
  *
  * Who needs it: code that runs where cudaMalloc is off limits - a real-time or

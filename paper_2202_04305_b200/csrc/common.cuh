@@ -120,3 +120,6 @@ sp_status sp_get_segment_ids(sp_tensor* t, cudaStream_t stream, const uint32_t**
 sp_status sp_get_merge_partition(sp_tensor* t, int64_t items_per_chunk, int64_t carry_elems_per_chunk,
                                  cudaStream_t stream, sp_partition* out);
 sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t nnz_per_chunk, cudaStream_t stream, sp_partition* out);
+
+// SpMV for rank-2 handles whose inner level is dense (dense_inner.cu).
+sp_status sp_spmv_dense_inner(const sp_tensor* A, const double* x, double* y, cudaStream_t stream);

@@ -467,6 +467,8 @@ bool matrix_encoding_ok(const sp_tensor* A) {
 
 extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* stream_) {
     if (!A || !x || !y) return SP_ERR_INVALID_ARG;
+    if (A->rank == 2 && A->lt[1] == SP_DENSE && A->ord[0] != A->ord[1])
+        return sp_spmv_dense_inner(A, x, y, static_cast<cudaStream_t>(stream_));
     if (!matrix_encoding_ok(A)) return SP_ERR_UNSUPPORTED;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const bool rowmajor = A->ord[0] == 0;

@@ -110,6 +110,11 @@ def test_row_band_spmv(oracle):
     x = I.uniform_pm1(0, 34, 65536)
     rows = np.array([0, 1, 499, 998, 999, 1000, 40000, 65535])
     ref, bd = oracle.spmv(65536, coo.coords[0], coo.coords[1], coo.vals, x, rows)
+    A = sp().sp_pack(coo.dims, coords, vals, (1, 0))          # CDR: the paper's best format for this input
+    assert A.nval == 1000 * 65536 and A.positions(0).cpu().numpy().tolist() == [0, 1000]
+    y = sp().sp_spmv(A, dev(x)).cpu().numpy()
+    assert_close(y[rows], ref, bd, "row band CDR")
+    assert np.all(y[1000:] == 0)
     for lt in [(0, 1), (1, 1)]:
         A = sp().sp_pack(coo.dims, coords, vals, lt)
         y = sp().sp_spmv(A, dev(x)).cpu().numpy()

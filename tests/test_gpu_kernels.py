@@ -39,6 +39,26 @@ def test_spmv(oracle, enc, name, coo):
     assert_close(y, ref, bd, f"spmv {enc} {name}")
 
 
+DENSE_INNER = {"CDR": ((1, 0), (0, 1)), "DD": ((0, 0), (0, 1)), "CDC": ((1, 0), (1, 0)), "DD-col": ((0, 0), (1, 0))}
+
+
+@pytest.mark.parametrize("enc", list(DENSE_INNER))
+@pytest.mark.parametrize("name,coo", MATS, ids=[m[0] for m in MATS])
+def test_spmv_dense_inner_level(oracle, enc, name, coo):
+    # (compressed, dense) is the paper's CDR (Section 6.2); explicit zeros in the stored slices add nothing
+    lt, od = DENSE_INNER[enc]
+    outer_dim = coo.dims[od[0]]
+    stored = outer_dim if lt[0] == 0 else np.unique(coo.coords[od[0]]).size
+    if stored * coo.dims[od[1]] > 1 << 24:
+        pytest.skip("dense slices too large to materialise")
+    coords, vals = to_dev(coo)
+    A = sp().sp_pack(coo.dims, coords, vals, lt, od)
+    x = I.uniform_pm1(11, 2, coo.dims[1])
+    y = sp().sp_spmv(A, dev(x)).cpu().numpy()
+    ref, bd = oracle.spmv(coo.dims[0], coo.coords[0], coo.coords[1], coo.vals, x)
+    assert_close(y, ref, bd, f"spmv {enc} {name}")
+
+
 @pytest.mark.parametrize("enc", list(MATRIX_ENCODINGS))
 @pytest.mark.parametrize("N", [1, 5, 32, 64, 70])
 @pytest.mark.parametrize("name,coo", MATS, ids=[m[0] for m in MATS])
@@ -106,7 +126,11 @@ def test_unsupported_encodings():
     coords, vals = to_dev(coo)
     A = b.sp_pack(coo.dims, coords, vals, (1, 0))
     with pytest.raises(b.SpError) as e:
-        b.sp_spmv(A, dev(np.ones(20)))
+        b.sp_spmm(A, dev(np.ones((20, 4))))
+    assert e.value.code == 2
+    T = b.sp_pack((20, 20, 1), coords + [coords[0] * 0], vals, (1, 1, 1))
+    with pytest.raises(b.SpError) as e:
+        b.sp_spmv(T, dev(np.ones(20)))
     assert e.value.code == 2
     S = b.sp_pack(coo.dims, coords, vals, (0, 1), (1, 0))
     with pytest.raises(b.SpError) as e:
