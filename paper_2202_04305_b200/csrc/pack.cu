@@ -371,6 +371,7 @@ struct EmitArgs {
     void* pos[SP_MAX_RANK];
     void* crd[SP_MAX_RANK];
     double* val;
+    uint32_t* seg_out;   // optional: level-0 coordinate of every stored entry (column-major matrices)
     bool pos64, crd64;
     unsigned flags;
     int* err;
@@ -450,6 +451,7 @@ __global__ void __launch_bounds__(kCtThreads) k_emit(EmitArgs a) {
             if (dup)
                 for (int64_t g = e + 1; g < a.n && a.keys[g] == k[i]; ++g) s += a.vals_in[a.idx[g]];
             a.val[ppos] = s;
+            if (a.seg_out) a.seg_out[ppos] = (uint32_t)(k[i] >> p.shift[0]);
         } else if (a.flags & SP_DUP_ERROR) {
             atomicOr(a.err, kErrDup);
         }
@@ -773,6 +775,16 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
         a.tileprefix = tileprefix; a.ntiles = ct_tiles;
         for (int l = 0; l < SP_MAX_RANK; ++l) { a.pos[l] = t->pos[l]; a.crd[l] = t->crd[l]; }
         a.val = t->val; a.pos64 = posBits == 64; a.crd64 = crdBits == 64; a.flags = flags; a.err = d_err;
+        // Column-major matrices run SpMM as a flat loop over entries and need each entry's column:
+        // it is in the sorted key anyway, so it is written here instead of being searched for later.
+        a.seg_out = nullptr;
+        if (rank == 2 && plan.src[0] == 1 && plan.lt[1] == SP_COMPRESSED && plan.sz[0] < ((int64_t)1 << 32)) {
+            sp_partition sg;
+            sg.aux = static_cast<int64_t*>(sp_dev_alloc((size_t)(t->nval ? t->nval : 1) * sizeof(uint32_t), stream));
+            if (!sg.aux) return fail(SP_ERR_ALLOC);
+            a.seg_out = reinterpret_cast<uint32_t*>(sg.aux);
+            t->parts[(uint64_t)SP_PART_SEGIDS << 56] = sg;
+        }
         k_emit<<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);
         sp_count_launches(1);
         for (int l = 0; l < rank; ++l) {
