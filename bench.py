@@ -247,12 +247,16 @@ def dist_barrier():
 
 
 # --------------------------------------------------------------------------- oracle arm / CPU baseline
-def oracle_sample(wl, small: bool):
+METRIC = ("f64 GFLOP/s of one pass of the sparse suite (per-kernel GFLOP/s, effective HBM GB/s and % of roofline "
+          "in `kernels`)")
+
+
+def oracle_sample(wl, small: bool, frac: int = 1):
     """Times the oracle, as it stands, on a bounded sample of every call of the step.
     Returns (seconds spent, extrapolated seconds for a full step, description)."""
     import oracle as O
     O.lib()
-    frac = 1          # the whole lists, except where a line below says otherwise (about 20 s of CPU work)
+    # frac = 1: the whole lists, except where a line below says otherwise (about 20 s of CPU work)
     c3, c2, c1b, c4, c5 = wl["c3"], wl["c2"], wl["c1b"], wl["c4"], wl["c5"]
     spent = 0.0
     full = 0.0
@@ -290,16 +294,18 @@ def run_reference(args, wl, model, total_flops, cfg):
     rank, _, world = dist_env()
     if rank != 0:
         return
+    # one full-list sample costs about 20 s of CPU; shrink it so that warm-up + steps stay near three minutes
+    frac = 1 if args.small else max(1, -(-20 * (args.steps + 1) // 180))
     for _ in range(min(args.warmup, 1)):
-        oracle_sample(wl, args.small)
+        oracle_sample(wl, args.small, frac)
     spent, full = [], []
     desc = ""
     for _ in range(args.steps):
-        s, f, desc = oracle_sample(wl, args.small)
+        s, f, desc = oracle_sample(wl, args.small, frac)
         spent.append(s); full.append(f)
     fstep = statistics.mean(full)
     val = total_flops / fstep / 1e9
-    line = {"impl": "reference", "metric": "f64 GFLOP/s of one pass of the sparse suite (CPU oracle, extrapolated from a bounded sample)",
+    line = {"impl": "reference", "metric": METRIC,
             "value": val, "unit": "GFLOP/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": statistics.mean(spent) * 1e3, "extrapolated_full_step_ms": fstep * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -438,7 +444,7 @@ def main():
                "sample": desc, "seconds_spent": round(spent, 2), "extrapolated_full_step_s": round(full, 2)}
 
     if rank == 0:
-        line = {"metric": "f64 GFLOP/s of one pass of the sparse suite (per-kernel GFLOP/s, effective HBM GB/s and % of roofline in `kernels`)",
+        line = {"metric": METRIC,
                 "value": round(value, 2), "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "f64", "data": "synthetic", "config": cfg, "clocks": clocks,

@@ -209,3 +209,35 @@ def test_mttkrp_exact_integers(oracle):
     for lt, od in TENSOR_ENCODINGS.values():
         T = sp().sp_pack(coo.dims, coords, vals, lt, od)
         assert np.array_equal(sp().sp_mttkrp(T, dev(B), dev(Cf)).cpu().numpy(), ref)
+
+
+@pytest.mark.parametrize("pb,cb,cbits", [(64, 64, 64), (32, 64, 32), (64, 32, 64), (0, 0, 32)])
+def test_every_kernel_with_wide_positions_and_coordinates(oracle, pb, cb, cbits):
+    # Section 4.1: pointer and index bit widths are part of the encoding; 0 means the native 64 bits
+    m = I.config2(seed=8, n=1200)
+    coords, vals = to_dev(m, cbits)
+    x = I.uniform_pm1(1, 2, 1200)
+    yref, yb = oracle.spmv(1200, m.coords[0], m.coords[1], m.vals, x)
+    for lt, od in list(MATRIX_ENCODINGS.values()) + [((1, 0), (0, 1))]:
+        A = sp().sp_pack(m.dims, coords, vals, lt, od, pb, cb)
+        assert A.pos_bits == (pb or 64) and A.crd_bits == (cb or 64)
+        assert_close(sp().sp_spmv(A, dev(x)).cpu().numpy(), yref, yb, f"spmv widths {pb}/{cb}")
+    A4, B4 = I.dense_operand(2, 8, 1200, 64), I.dense_operand(2, 9, 64, 1200)
+    xe, be = oracle.sddmm(m.coords[0], m.coords[1], m.vals, A4, B4)
+    for lt in [(0, 1), (1, 1)]:
+        S = sp().sp_pack(m.dims, coords, vals, lt, None, pb, cb)
+        ep = oracle.pack(m.dims, m.coords, m.vals, lt).entry_pos
+        ref = np.empty_like(xe); bd = np.empty_like(be)
+        ref[ep] = xe; bd[ep] = be
+        assert_close(sp().sp_sddmm(S, dev(A4), dev(B4)).cpu().numpy(), ref, bd, f"sddmm widths {pb}/{cb}")
+    t = I.config5(seed=9, dim=96, nnz=15000)
+    tc, tv = to_dev(t, cbits)
+    Bf, Cf = I.dense_operand(3, 10, 96, 32), I.dense_operand(3, 11, 96, 32)
+    Mref, Mb = oracle.mttkrp(96, *t.coords, t.vals, Bf, Cf)
+    for lt, od in TENSOR_ENCODINGS.values():
+        T = sp().sp_pack(t.dims, tc, tv, lt, od, pb, cb)
+        assert_close(sp().sp_mttkrp(T, dev(Bf), dev(Cf)).cpu().numpy(), Mref, Mb, f"mttkrp widths {pb}/{cb}")
+        for R in (5,):      # the generic (odd R) kernel as well
+            B5, C5 = I.dense_operand(3, 12, 96, R), I.dense_operand(3, 13, 96, R)
+            r5, b5 = oracle.mttkrp(96, *t.coords, t.vals, B5, C5)
+            assert_close(sp().sp_mttkrp(T, dev(B5), dev(C5)).cpu().numpy(), r5, b5, f"mttkrp R=5 widths {pb}/{cb}")
