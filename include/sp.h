@@ -40,7 +40,7 @@
 extern "C" {
 #endif
 
-#define SP_MAX_RANK 3
+#define SP_MAX_RANK 5
 
 typedef struct sp_tensor sp_tensor;   /* opaque; owns device arrays */
 

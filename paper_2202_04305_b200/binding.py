@@ -12,6 +12,7 @@ import os
 import torch
 
 DENSE, COMPRESSED = 0, 1
+MAX_RANK = 5
 DUP_SUM, DUP_ERROR = 0, 1
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -106,9 +107,9 @@ class SpTensor:
     def __init__(self, handle):
         self._h = handle
         rank = C.c_int()
-        dims = (C.c_int64 * 3)()
-        lt = (C.c_int * 3)()
-        od = (C.c_int * 3)()
+        dims = (C.c_int64 * MAX_RANK)()
+        lt = (C.c_int * MAX_RANK)()
+        od = (C.c_int * MAX_RANK)()
         pb, cb = C.c_int(), C.c_int()
         _check(_lib.sp_info(self._h, C.byref(rank), dims, lt, od, C.byref(pb), C.byref(cb)), "sp_info")
         self.rank = rank.value

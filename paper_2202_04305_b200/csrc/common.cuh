@@ -27,14 +27,14 @@ struct sp_partition {
 
 struct sp_tensor {
     int rank = 0;
-    int64_t dims[SP_MAX_RANK] = {0, 0, 0};
-    int lt[SP_MAX_RANK] = {0, 0, 0};
-    int ord[SP_MAX_RANK] = {0, 1, 2};
+    int64_t dims[SP_MAX_RANK] = {};
+    int lt[SP_MAX_RANK] = {};
+    int ord[SP_MAX_RANK] = {};
     int posBits = 64, crdBits = 64;
-    void* pos[SP_MAX_RANK] = {nullptr, nullptr, nullptr};
-    int64_t npos[SP_MAX_RANK] = {0, 0, 0};
-    void* crd[SP_MAX_RANK] = {nullptr, nullptr, nullptr};
-    int64_t ncrd[SP_MAX_RANK] = {0, 0, 0};
+    void* pos[SP_MAX_RANK] = {};
+    int64_t npos[SP_MAX_RANK] = {};
+    void* crd[SP_MAX_RANK] = {};
+    int64_t ncrd[SP_MAX_RANK] = {};
     double* val = nullptr;
     int64_t nval = 0;
     int device = 0;

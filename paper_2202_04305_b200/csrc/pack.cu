@@ -69,18 +69,18 @@ struct LevelPlan {
 };
 
 // ------------------------------------------------------------------ keys ---
+struct LevelCoords { const void* p[SP_MAX_RANK]; };   // coordinate array of the dimension stored at level l
+
 template <typename CT>
-__global__ void k_build_keys(const CT* c0, const CT* c1, const CT* c2, int64_t n, LevelPlan p,
-                             uint64_t* keys, uint32_t* idx, int* err) {
+__global__ void k_build_keys(LevelCoords lc, int64_t n, LevelPlan p, uint64_t* keys, uint32_t* idx, int* err) {
     int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (e >= n) return;
-    const CT* src[SP_MAX_RANK] = {c0, c1, c2};
     uint64_t key = 0;
     bool bad = false;
 #pragma unroll
     for (int l = 0; l < SP_MAX_RANK; ++l) {
         if (l < p.rank) {
-            CT c = src[p.src[l]][e];
+            CT c = static_cast<const CT*>(lc.p[l])[e];
             if (c < 0 || (int64_t)c >= p.sz[l]) { bad = true; c = 0; }
             key |= (uint64_t)c << p.shift[l];
         }
@@ -282,7 +282,7 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
 constexpr int kCtThreads = 256;
 constexpr int kCtIpt = 8;
 constexpr int kCtTile = kCtThreads * kCtIpt;   // 2048
-constexpr int kField = 21;                     // three 21-bit counters packed in 64 bits
+constexpr int kField = 12;                     // SP_MAX_RANK 12-bit counters (a tile has 2048 entries) in 64 bits
 constexpr uint64_t kFieldMask = (1ull << kField) - 1;
 
 __device__ __forceinline__ uint64_t level_flags(uint64_t k, uint64_t kprev, bool first, const LevelPlan& p) {
@@ -339,25 +339,26 @@ k_count_flags(const uint64_t* __restrict__ keys, int64_t n, LevelPlan p, uint64_
     if (threadIdx.x == 0) tilesum[blockIdx.x] = tot;
 }
 
+static_assert(kField * SP_MAX_RANK <= 64 && (1 << kField) > kCtTile, "packed per-tile counters");
+
 // Single block (512 threads): tilesum (packed) -> tileprefix[l][tile] (exclusive), counts[l].
+// Across tiles the counts outgrow the packed fields, so each level is scanned on its own.
 __global__ void __launch_bounds__(512)
-k_scan_tiles(const uint64_t* __restrict__ tilesum, int64_t ntiles, int64_t* __restrict__ tileprefix,
+k_scan_tiles(const uint64_t* __restrict__ tilesum, int64_t ntiles, int rank, int64_t* __restrict__ tileprefix,
              int64_t* __restrict__ counts) {
     __shared__ uint64_t sums[16];
-    int64_t run[SP_MAX_RANK] = {0, 0, 0};
-    for (int64_t base = 0; base < ntiles; base += 512) {
-        int64_t i = base + threadIdx.x;
-        uint64_t v = i < ntiles ? tilesum[i] : 0;
-        uint64_t tot;
-        uint64_t ex = block_excl_scan64(v, sums, &tot);
-#pragma unroll
-        for (int l = 0; l < SP_MAX_RANK; ++l) {
-            if (i < ntiles) tileprefix[(int64_t)l * ntiles + i] = run[l] + (int64_t)((ex >> (kField * l)) & kFieldMask);
-            run[l] += (int64_t)((tot >> (kField * l)) & kFieldMask);
+    for (int l = 0; l < rank; ++l) {
+        uint64_t run = 0;
+        for (int64_t base = 0; base < ntiles; base += 512) {
+            const int64_t i = base + threadIdx.x;
+            const uint64_t v = i < ntiles ? ((tilesum[i] >> (kField * l)) & kFieldMask) : 0;
+            uint64_t tot;
+            const uint64_t ex = block_excl_scan64(v, sums, &tot);
+            if (i < ntiles) tileprefix[(int64_t)l * ntiles + i] = (int64_t)(run + ex);
+            run += tot;
         }
+        if (threadIdx.x == 0) counts[l] = (int64_t)run;
     }
-    if (threadIdx.x == 0)
-        for (int l = 0; l < SP_MAX_RANK; ++l) counts[l] = run[l];
 }
 
 struct EmitArgs {
@@ -403,7 +404,7 @@ __global__ void __launch_bounds__(kCtThreads) k_emit(EmitArgs a) {
     int64_t incl[SP_MAX_RANK];
 #pragma unroll
     for (int l = 0; l < SP_MAX_RANK; ++l)
-        incl[l] = a.tileprefix[(int64_t)l * a.ntiles + blockIdx.x] + (int64_t)((ex >> (kField * l)) & kFieldMask);
+        incl[l] = l < p.rank ? a.tileprefix[(int64_t)l * a.ntiles + blockIdx.x] + (int64_t)((ex >> (kField * l)) & kFieldMask) : 0;
 
     // values of this thread's entries, gathered before the (sequential) level walk needs them
     uint32_t id[kCtIpt];
@@ -626,7 +627,7 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
     LevelPlan plan;
     memset(&plan, 0, sizeof plan);
     plan.rank = rank;
-    bool seen[SP_MAX_RANK] = {false, false, false};
+    bool seen[SP_MAX_RANK] = {};
     int total_bits = 0;
     for (int l = 0; l < rank; ++l) {
         int d = dimOrdering ? dimOrdering[l] : l;
@@ -653,7 +654,7 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
     PhaseTimer timer(stream, g_profiling);
     int npasses_done = 0;
     const int64_t n = nnz;
-    int64_t counts[SP_MAX_RANK] = {0, 0, 0};
+    int64_t counts[SP_MAX_RANK] = {};
     uint64_t* keys = nullptr;
     uint32_t* idx = nullptr;
     int64_t* tileprefix = nullptr;
@@ -674,15 +675,11 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
         if (ws.failed) return SP_ERR_ALLOC;
         SP_CUDA(cudaMemsetAsync(d_err, 0, sizeof(int), stream));
 
-        const void* c[SP_MAX_RANK] = {coo_coords[0], rank > 1 ? coo_coords[1] : coo_coords[0],
-                                      rank > 2 ? coo_coords[2] : coo_coords[0]};
+        LevelCoords lc;
+        for (int l = 0; l < SP_MAX_RANK; ++l) lc.p[l] = coo_coords[l < rank ? plan.src[l] : 0];
         const unsigned kb = (unsigned)sp_ceil_div(n, 256);
-        if (coo_coord_bits == 32)
-            k_build_keys<int32_t><<<kb, 256, 0, stream>>>((const int32_t*)c[0], (const int32_t*)c[1],
-                                                          (const int32_t*)c[2], n, plan, kbuf[0], ibuf[0], d_err);
-        else
-            k_build_keys<int64_t><<<kb, 256, 0, stream>>>((const int64_t*)c[0], (const int64_t*)c[1],
-                                                          (const int64_t*)c[2], n, plan, kbuf[0], ibuf[0], d_err);
+        if (coo_coord_bits == 32) k_build_keys<int32_t><<<kb, 256, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], d_err);
+        else k_build_keys<int64_t><<<kb, 256, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], d_err);
         SP_LAUNCH_CHECK();
         sp_count_launches(1);
         timer.mark(kPhKeys);
@@ -710,7 +707,7 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
         idx = ibuf[cur];
 
         k_count_flags<<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum);
-        k_scan_tiles<<<1, 512, 0, stream>>>(tilesum, ct_tiles, tileprefix, d_counts);
+        k_scan_tiles<<<1, 512, 0, stream>>>(tilesum, ct_tiles, rank, tileprefix, d_counts);
         SP_LAUNCH_CHECK();
         timer.mark(kPhCount);
         sp_count_launches(3);
@@ -731,7 +728,7 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
     const size_t pw = posBits / 8, cw = crdBits / 8;
     sp_status st = SP_OK;
     int64_t parents = 1;
-    int64_t parents_at[SP_MAX_RANK] = {0, 0, 0};
+    int64_t parents_at[SP_MAX_RANK] = {};
     for (int l = 0; l < rank && st == SP_OK; ++l) {
         t->dims[l] = dims[l];
         t->lt[l] = plan.lt[l];
@@ -762,7 +759,7 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
 
     const bool trailing_dense = plan.lt[rank - 1] == SP_DENSE;
     if (trailing_dense && t->nval > 0) SP_CUDA_T(cudaMemsetAsync(t->val, 0, (size_t)t->nval * sizeof(double), stream));
-    bool needs_fill[SP_MAX_RANK] = {false, false, false};
+    bool needs_fill[SP_MAX_RANK] = {};
     for (int l = 0; l < rank; ++l) {
         if (plan.lt[l] != SP_COMPRESSED) continue;
         needs_fill[l] = n > 0 && l >= 1 && plan.lt[l - 1] == SP_DENSE;

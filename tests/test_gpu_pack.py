@@ -134,3 +134,45 @@ def test_pack_is_repeatable():
         assert np.array_equal(a.positions(l).cpu().numpy(), b.positions(l).cpu().numpy())
         assert np.array_equal(a.coordinates(l).cpu().numpy(), b.coordinates(l).cpu().numpy())
     assert np.array_equal(a.values().cpu().numpy(), b.values().cpu().numpy())
+
+
+def test_rank_four_every_encoding(oracle):
+    dims = (5, 3, 6, 4)
+    coo = I.uniform_tensor(dims, 97, seed=44)
+    coords, vals = to_dev(coo)
+    n = 0
+    for lt, od in all_encodings(4):
+        t = sp().sp_pack(dims, coords, vals, lt, od)
+        assert_storage_equal(t, oracle.pack(dims, coo.coords, coo.vals, lt, od))
+        n += 1
+    assert n == 2 ** 4 * 24
+
+
+def test_rank_five_sampled_encodings_and_round_trip(oracle):
+    dims = (4, 3, 2, 5, 3)
+    coo = I.uniform_tensor(dims, 150, seed=45)
+    coords, vals = to_dev(coo, 64)
+    for n, (lt, od) in enumerate(all_encodings(5)):
+        if n % 53:
+            continue
+        t = sp().sp_pack(dims, coords, vals, lt, od, 64, 32)
+        ref = oracle.pack(dims, coo.coords, coo.vals, lt, od)
+        assert_storage_equal(t, ref)
+        oc, ov = sp().sp_unpack(t)
+        rc, rv = oracle.unpack(ref)
+        for d in range(5):
+            assert np.array_equal(oc[d].cpu().numpy(), rc[d])
+        assert np.array_equal(ov.cpu().numpy(), rv)
+
+
+@pytest.mark.parametrize("dims,nnz", [((183, 24, 1140, 1717), 300_000), ((165427, 11374, 2, 100, 89), 400_000)])
+def test_all_compressed_four_and_five_dimensional_shapes(oracle, dims, nnz):
+    # the shapes (not the contents) of the 4-d and 5-d tensors whose packing Table 1 times; uniform entries stand in
+    coo = I.uniform_tensor(dims, nnz, seed=len(dims))
+    coords, vals = to_dev(coo)
+    lt = (1,) * len(dims)
+    t = sp().sp_pack(dims, coords, vals, lt)
+    assert_storage_equal(t, oracle.pack(dims, coo.coords, coo.vals, lt))
+    od = tuple(reversed(range(len(dims))))
+    t = sp().sp_pack(dims, coords, vals, lt, od)
+    assert_storage_equal(t, oracle.pack(dims, coo.coords, coo.vals, lt, od))

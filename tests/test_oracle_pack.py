@@ -55,7 +55,8 @@ def _dense_of(dims, coords, vals):
     return d
 
 
-@pytest.mark.parametrize("dims,nnz", [((7,), 3), ((6, 5), 11), ((5, 8), 0), ((4, 3, 5), 17), ((3, 3, 4), 36)])
+@pytest.mark.parametrize("dims,nnz", [((7,), 3), ((6, 5), 11), ((5, 8), 0), ((4, 3, 5), 17), ((3, 3, 4), 36),
+                                      ((3, 2, 4, 3), 19)])
 def test_round_trip_dense_brute_force_all_encodings(oracle, dims, nnz):
     rank = len(dims)
     coo = I.uniform_tensor(dims, nnz, seed=rank + nnz)
