@@ -144,7 +144,8 @@ sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* stream);
 /*
  * sp_spmm - C[i,j] = sum_k A[i,k] * B[k,j], A sparse, B and C dense
  * (Sections 1 and 5.2).  B is dims[1] x N with leading dimension ldb, C is
- * dims[0] x N with ldc.  Encodings and the atomics remark as for sp_spmv.
+ * dims[0] x N with ldc.  Encodings (all eight two-dimensional ones, the set the
+ * search loop of Section 5.2 enumerates) and the atomics remark as for sp_spmv.
  */
 sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t ldb,
                   double* C, int64_t ldc, void* stream);

@@ -123,3 +123,5 @@ sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t nnz_per_chunk, cudaStrea
 
 // SpMV for rank-2 handles whose inner level is dense (dense_inner.cu).
 sp_status sp_spmv_dense_inner(const sp_tensor* A, const double* x, double* y, cudaStream_t stream);
+sp_status sp_spmm_dense_inner(const sp_tensor* A, const double* B, int64_t N, int64_t ldb, double* C, int64_t ldc,
+                              cudaStream_t stream);

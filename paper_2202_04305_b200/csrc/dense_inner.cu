@@ -1,4 +1,4 @@
-// SpMV over encodings whose inner level is dense: (compressed, dense) - the paper's "CDR" of
+// SpMV and SpMM over encodings whose inner level is dense: (compressed, dense) - the paper's "CDR" of
 // Section 6.2, the best format for its row-band matrices - and (dense, dense), in either order.
 //
 // values holds one full inner slice per stored outer index q (explicit zeros included), so the
@@ -82,6 +82,76 @@ k_spmv_dense_cols(const double* __restrict__ val, const I* __restrict__ outer, i
     atomicAdd(y + i, s);
 }
 
+// SpMM with a dense inner level: C[i,:] = sum_k A[i,k] * B[k,:] where A's stored slices are dense.
+// A block owns kRT output rows and one 32-column tile of C and walks the contraction index in steps of
+// kKT: the kRT x kKT tile of A is staged in shared memory (stored [k][row], so a warp reads its four
+// row values with one 32-byte broadcast), each warp owns 4 rows, lane = column, and every B row is
+// loaded once per warp and used for 4 rows.
+//   row-major    : output row = stored slice q (i = crd[0][q]), k = inner index,  A[q,k]  = val[q*inner + k]
+//   column-major : output row = inner index i,  k = stored slice q (crd[0][q]),   A[i,q]  = val[q*inner + i]
+constexpr int kRT = 32, kKT = 32;
+
+template <typename I, bool ROWMAJOR>
+__global__ void __launch_bounds__(kDThreads)
+k_spmm_dense_inner(const double* __restrict__ val, const I* __restrict__ outer, int64_t nslices, int64_t inner,
+                   const double* __restrict__ B, int64_t N, int64_t ldb, double* __restrict__ C, int64_t ldc,
+                   int64_t kchunk) {
+    __shared__ double s_a[kKT][kRT + 4];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t nrows = ROWMAJOR ? nslices : inner;     // output rows this kernel produces
+    const int64_t nk = ROWMAJOR ? inner : nslices;        // length of the contraction
+    const int64_t r0 = (int64_t)blockIdx.x * kRT;
+    const int64_t col = (int64_t)blockIdx.y * 32 + lane;
+    const bool on = col < N;
+    const double* Bc = B + (on ? col : (int64_t)blockIdx.y * 32);
+    double acc[4] = {0.0, 0.0, 0.0, 0.0};
+    // blockIdx.z owns the contraction range [kbeg, kend); with more than one range the partial
+    // products are added into C (zeroed by the caller) with atomics
+    const int64_t kbeg = (int64_t)blockIdx.z * kchunk;
+    const int64_t kend = kbeg + kchunk < nk ? kbeg + kchunk : nk;
+    for (int64_t k0 = kbeg; k0 < kend; k0 += kKT) {
+        __syncthreads();
+        // stage A[r0 .. r0+kRT) x [k0 .. k0+kKT), zero outside
+        for (int e = threadIdx.x; e < kRT * kKT; e += kDThreads) {
+            // the fast index of the load follows the contiguous index of val
+            const int rr = ROWMAJOR ? e / kKT : e % kRT;
+            const int kk = ROWMAJOR ? e % kKT : e / kRT;
+            const int64_t r = r0 + rr, k = k0 + kk;
+            double a = 0.0;
+            if (r < nrows && k < kend) a = ROWMAJOR ? __ldcs(val + r * inner + k) : __ldcs(val + k * inner + r);
+            s_a[kk][rr] = a;
+        }
+        __syncthreads();
+        const int kmax = (int)(kend - k0 < kKT ? kend - k0 : kKT);
+        double b[kKT / 4];
+        for (int kb = 0; kb < kmax; kb += kKT / 4) {      // 8 B rows in flight per warp
+#pragma unroll
+            for (int u = 0; u < kKT / 4; ++u) {
+                const int64_t k = k0 + kb + u;
+                const int64_t krow = k < nk ? (ROWMAJOR ? k : (outer ? (int64_t)outer[k] : k)) : 0;
+                b[u] = __ldg(Bc + krow * ldb);
+            }
+#pragma unroll
+            for (int u = 0; u < kKT / 4; ++u) {
+                if (kb + u < kmax) {
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) acc[r] = fma(s_a[kb + u][4 * w + r], b[u], acc[r]);
+                }
+            }
+        }
+    }
+    if (on) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int64_t row = r0 + 4 * w + r;
+            if (row < nrows) {
+                double* dst = C + (ROWMAJOR ? (outer ? (int64_t)outer[row] : row) : row) * ldc + col;
+                if (gridDim.z > 1) atomicAdd(dst, acc[r]); else *dst = acc[r];
+            }
+        }
+    }
+}
+
 }  // namespace
 
 // Called by sp_spmv for rank-2 handles whose level 1 is dense.
@@ -114,6 +184,52 @@ sp_status sp_spmv_dense_inner(const sp_tensor* A, const double* x, double* y, cu
     } while (0)
     if (A->crdBits == 32) SP_DENSE_LAUNCH(uint32_t); else SP_DENSE_LAUNCH(uint64_t);
 #undef SP_DENSE_LAUNCH
+    SP_LAUNCH_CHECK();
+    sp_count_launches(1);
+    return SP_OK;
+}
+
+// Called by sp_spmm for rank-2 handles whose level 1 is dense.
+sp_status sp_spmm_dense_inner(const sp_tensor* A, const double* B, int64_t N, int64_t ldb, double* C, int64_t ldc,
+                              cudaStream_t stream) {
+    const bool rowmajor = A->ord[0] == 0;
+    const bool outer_c = A->lt[0] == SP_COMPRESSED;
+    const int64_t inner = A->dims[A->ord[1]];
+    const int64_t nslices = outer_c ? A->ncrd[0] : A->dims[A->ord[0]];
+    const int64_t m = A->dims[0];
+    if (nslices == 0 || inner == 0) {                  // nothing stored: the product is zero
+        if (ldc == N) SP_CUDA(cudaMemsetAsync(C, 0, (size_t)m * N * sizeof(double), stream));
+        else SP_CUDA(cudaMemset2DAsync(C, (size_t)ldc * sizeof(double), 0, (size_t)N * sizeof(double), (size_t)m, stream));
+        return SP_OK;
+    }
+    const int64_t nrows = rowmajor ? nslices : inner;
+    const int64_t nk = rowmajor ? inner : nslices;
+    const int64_t rb = sp_ceil_div(nrows, kRT), cb = sp_ceil_div(N, 32);
+    // few row blocks and a long contraction (a row band): split the contraction so every SM has work
+    int64_t ksplit = 1;
+    if (rb * cb < 4 * 148) {
+        ksplit = sp_ceil_div(4 * 148, rb * cb);
+        const int64_t most = sp_ceil_div(nk, 8 * kKT);
+        if (ksplit > most) ksplit = most;
+        if (ksplit > 65535) ksplit = 65535;
+        if (ksplit < 1) ksplit = 1;
+    }
+    const int64_t kchunk = sp_ceil_div(sp_ceil_div(nk, ksplit), kKT) * kKT;
+    ksplit = sp_ceil_div(nk, kchunk);
+    if ((rowmajor && outer_c) || ksplit > 1) {          // rows not stored are zero; split sums start at zero
+        if (ldc == N) SP_CUDA(cudaMemsetAsync(C, 0, (size_t)m * N * sizeof(double), stream));
+        else SP_CUDA(cudaMemset2DAsync(C, (size_t)ldc * sizeof(double), 0, (size_t)N * sizeof(double), (size_t)m, stream));
+    }
+    if (cb > 65535) return SP_ERR_UNSUPPORTED;
+    dim3 grid((unsigned)rb, (unsigned)cb, (unsigned)(ksplit > 0 ? ksplit : 1));
+#define SP_DENSE_MM(I)                                                                                                  \
+    do {                                                                                                                \
+        const I* outer = outer_c ? static_cast<const I*>(A->crd[0]) : nullptr;                                          \
+        if (rowmajor) k_spmm_dense_inner<I, true><<<grid, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, B, N, ldb, C, ldc, kchunk); \
+        else k_spmm_dense_inner<I, false><<<grid, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, B, N, ldb, C, ldc, kchunk);       \
+    } while (0)
+    if (A->crdBits == 32) SP_DENSE_MM(uint32_t); else SP_DENSE_MM(uint64_t);
+#undef SP_DENSE_MM
     SP_LAUNCH_CHECK();
     sp_count_launches(1);
     return SP_OK;

@@ -504,8 +504,10 @@ extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* str
 extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t ldb, double* C, int64_t ldc,
                              void* stream_) {
     if (!A || !B || !C || N < 1 || ldb < N || ldc < N) return SP_ERR_INVALID_ARG;
-    if (!matrix_encoding_ok(A)) return SP_ERR_UNSUPPORTED;
     if (N >= (1 << 20)) return SP_ERR_UNSUPPORTED;
+    if (A->rank == 2 && A->lt[1] == SP_DENSE && A->ord[0] != A->ord[1])
+        return sp_spmm_dense_inner(A, B, N, ldb, C, ldc, static_cast<cudaStream_t>(stream_));
+    if (!matrix_encoding_ok(A)) return SP_ERR_UNSUPPORTED;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const bool rowmajor = A->ord[0] == 0;
     const bool dbl = A->lt[0] == SP_COMPRESSED;

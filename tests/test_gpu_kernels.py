@@ -59,6 +59,22 @@ def test_spmv_dense_inner_level(oracle, enc, name, coo):
     assert_close(y, ref, bd, f"spmv {enc} {name}")
 
 
+@pytest.mark.parametrize("enc", list(DENSE_INNER))
+@pytest.mark.parametrize("N", [1, 7, 32, 70])
+@pytest.mark.parametrize("name,coo", MATS, ids=[m[0] for m in MATS])
+def test_spmm_dense_inner_level(oracle, enc, N, name, coo):
+    lt, od = DENSE_INNER[enc]
+    stored = coo.dims[od[0]] if lt[0] == 0 else np.unique(coo.coords[od[0]]).size
+    if stored * coo.dims[od[1]] > 1 << 22 or (N in (7, 70) and name not in ("uniform", "band", "tiny")):
+        pytest.skip("dense slices too large, or ragged width covered elsewhere")
+    coords, vals = to_dev(coo)
+    A = sp().sp_pack(coo.dims, coords, vals, lt, od)
+    B = I.dense_operand(12, 3, coo.dims[1], N)
+    Cg = sp().sp_spmm(A, dev(B)).cpu().numpy()
+    ref, bd = oracle.spmm(coo.dims[0], coo.coords[0], coo.coords[1], coo.vals, B)
+    assert_close(Cg, ref, bd, f"spmm {enc} {name} N={N}")
+
+
 @pytest.mark.parametrize("enc", list(MATRIX_ENCODINGS))
 @pytest.mark.parametrize("N", [1, 5, 32, 64, 70])
 @pytest.mark.parametrize("name,coo", MATS, ids=[m[0] for m in MATS])
@@ -126,7 +142,7 @@ def test_unsupported_encodings():
     coords, vals = to_dev(coo)
     A = b.sp_pack(coo.dims, coords, vals, (1, 0))
     with pytest.raises(b.SpError) as e:
-        b.sp_spmm(A, dev(np.ones((20, 4))))
+        b.sp_sddmm(A, dev(np.ones((20, 4))), dev(np.ones((4, 20))))
     assert e.value.code == 2
     T = b.sp_pack((20, 20, 1), coords + [coords[0] * 0], vals, (1, 1, 1))
     with pytest.raises(b.SpError) as e:
