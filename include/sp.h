@@ -152,8 +152,8 @@ sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t ldb,
 
 /*
  * sp_sddmm - X[i,j] = S[i,j] * sum_k A[i,k] * B[k,j] for the stored (i,j) of
- * S (Section 6.2).  S: rank 2, (dense|compressed, compressed), identity
- * ordering.  A is dims[0] x K (lda), B is K x dims[1] (ldb).  x_vals receives
+ * S (Section 6.2).  S: rank 2, (dense|compressed, compressed), either
+ * ordering (CSR, DCSR, CSC, DCSC).  A is dims[0] x K (lda), B is K x dims[1] (ldb).  x_vals receives
  * one value per stored entry of S, in S's storage order (X shares S's
  * positions and coordinates); its length is sp_values' len.
  */
@@ -170,6 +170,17 @@ sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const double* B, 
  */
 sp_status sp_mttkrp(sp_tensor* T, const double* B, const double* C, int64_t R,
                     double* M, void* stream);
+
+/*
+ * sp_mttkrp_mode - the same product for any output dimension:
+ *   M[c_mode, r] = sum over the other two coordinates of T[c0,c1,c2] * F_a[c_a, r] * F_b[c_b, r]
+ * (Section 6.3 gives the mode-0 case).  T must store logical dimension `mode` at
+ * level 0 (pack it with that dimOrdering), levels 1 and 2 compressed.
+ * factors: host array of 3 device pointers, factors[d] being the dims[d] x R
+ * matrix of dimension d; factors[mode] is ignored.  M is dims[mode] x R.
+ */
+sp_status sp_mttkrp_mode(sp_tensor* T, int mode, const double* const* factors, int64_t R,
+                         double* M, void* stream);
 
 /*
  * sp_spmv_static - y = A * x exactly as sp_spmv computes it (same kernels, same

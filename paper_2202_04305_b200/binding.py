@@ -20,7 +20,7 @@ _LIB_PATH = os.path.join(_HERE, "libsp.so")
 
 SYMBOLS = ["sp_status_string", "sp_set_allocator", "sp_pack", "sp_free", "sp_info", "sp_positions",
            "sp_coordinates", "sp_values", "sp_unpack", "sp_spmv", "sp_spmm", "sp_sddmm", "sp_mttkrp",
-           "sp_set_profiling", "sp_get_pack_profile", "sp_launch_count", "sp_spmv_static"]
+           "sp_set_profiling", "sp_get_pack_profile", "sp_launch_count", "sp_spmv_static", "sp_mttkrp_mode"]
 SPMV_STATIC_MAX_ITEMS = 134217728
 
 
@@ -259,3 +259,18 @@ def sp_get_pack_profile():
     n = C.c_int()
     _check(_lib.sp_get_pack_profile(ms, C.byref(n)), "sp_get_pack_profile")
     return {k: ms[i] for i, k in enumerate(PACK_PHASES)}, n.value
+
+
+def sp_mttkrp_mode(T: SpTensor, mode: int, factors, M=None):
+    """factors: three CUDA float64 matrices (factors[mode] may be None); T stores dimension `mode` at level 0."""
+    use = [f for d, f in enumerate(factors) if d != mode]
+    for f in use:
+        _f64(f, "factor")
+        if not f.is_contiguous():
+            raise ValueError("factor matrices must be contiguous")
+    R = use[0].shape[1]
+    if M is None:
+        M = torch.empty((T.dims[mode], R), dtype=torch.float64, device="cuda")
+    ptrs = (C.c_void_p * 3)(*[f.data_ptr() if (f is not None and d != mode) else 0 for d, f in enumerate(factors)])
+    _check(_lib.sp_mttkrp_mode(T._h, C.c_int(mode), ptrs, C.c_int64(R), _dptr(M), _stream()), "sp_mttkrp_mode")
+    return M

@@ -386,17 +386,35 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
 
 }  // namespace
 
+// F1 / F2: factor matrices of the dimensions stored at levels 1 / 2; M: rows of the level-0 dimension.
+static sp_status mttkrp_levels(sp_tensor* T, const double* F1, const double* F2, int64_t R, double* M, cudaStream_t stream);
+
 extern "C" sp_status sp_mttkrp(sp_tensor* T, const double* B, const double* C, int64_t R, double* M, void* stream_) {
     if (!T || !B || !C || !M || R < 1) return SP_ERR_INVALID_ARG;
     if (T->rank != 3 || T->ord[0] != 0 || T->lt[1] != SP_COMPRESSED || T->lt[2] != SP_COMPRESSED)
         return SP_ERR_UNSUPPORTED;
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    SP_CUDA(cudaMemsetAsync(M, 0, (size_t)T->dims[0] * R * sizeof(double), stream));
+    return mttkrp_levels(T, T->ord[1] == 1 ? B : C, T->ord[1] == 1 ? C : B, R, M, static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" sp_status sp_mttkrp_mode(sp_tensor* T, int mode, const double* const* factors, int64_t R, double* M,
+                                    void* stream_) {
+    if (!T || !factors || !M || R < 1 || mode < 0 || mode > 2) return SP_ERR_INVALID_ARG;
+    if (T->rank != 3 || T->ord[0] != mode || T->lt[1] != SP_COMPRESSED || T->lt[2] != SP_COMPRESSED)
+        return SP_ERR_UNSUPPORTED;
+    const double* F1 = factors[T->ord[1]];
+    const double* F2 = factors[T->ord[2]];
+    if (!F1 || !F2) return SP_ERR_INVALID_ARG;
+    return mttkrp_levels(T, F1, F2, R, M, static_cast<cudaStream_t>(stream_));
+}
+
+static sp_status mttkrp_levels(sp_tensor* T, const double* F1, const double* F2, int64_t R, double* M, cudaStream_t stream) {
+    const double* B = F1;
+    const double* C = F2;
+    SP_CUDA(cudaMemsetAsync(M, 0, (size_t)T->dims[T->ord[0]] * R * sizeof(double), stream));
     const int64_t nnz = T->ncrd[2];
     if (nnz == 0) return SP_OK;
-    const double* F1 = T->ord[1] == 1 ? B : C;   // factor of the dimension kept at level 1
-    const double* F2 = T->ord[1] == 1 ? C : B;
-    const int64_t maxdim = T->dims[1] > T->dims[2] ? T->dims[1] : T->dims[2];
+    const int64_t d1 = T->dims[T->ord[1]], d2 = T->dims[T->ord[2]];
+    const int64_t maxdim = d1 > d2 ? d1 : d2;
     const bool fast = (R % 2 == 0) && maxdim * R < ((int64_t)1 << 31) && reinterpret_cast<uintptr_t>(B) % 16 == 0 &&
                       reinterpret_cast<uintptr_t>(C) % 16 == 0 && reinterpret_cast<uintptr_t>(M) % 16 == 0;
     sp_partition part;

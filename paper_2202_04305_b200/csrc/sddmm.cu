@@ -1,5 +1,5 @@
 // sp_sddmm: X[i,j] = S[i,j] * sum_k A[i,k] * B[k,j] over the stored (i,j) of S
-// (Section 6.2), S in (dense|compressed, compressed) row-major storage.
+// (Section 6.2), S in (dense|compressed, compressed) storage, row- or column-major.
 //
 // Loop shape: for each stored row i, for each p in pos[1][q]..pos[1][q+1]:
 // j = crd[1][p]; x[p] = S.val[p] * dot(A[i,:], B[:,j]).  B is given K x n row-major,
@@ -133,7 +133,8 @@ k_sddmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __re
 extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const double* B, int64_t ldb, int64_t K,
                               double* x_vals, void* stream_) {
     if (!S || !A || !B || K < 1 || lda < K) return SP_ERR_INVALID_ARG;
-    if (S->rank != 2 || S->lt[1] != SP_COMPRESSED || S->ord[0] != 0 || S->ord[1] != 1) return SP_ERR_UNSUPPORTED;
+    if (S->rank != 2 || S->lt[1] != SP_COMPRESSED || S->ord[0] == S->ord[1]) return SP_ERR_UNSUPPORTED;
+    const bool colmajor = S->ord[0] == 1;      // S stored by columns (CSC, DCSC)
     const int64_t n = S->dims[1];
     if (ldb < n) return SP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -144,6 +145,7 @@ extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const 
 
     sp_workspace ws(stream);
     const int64_t ldt = (K + 1) & ~(int64_t)1;   // even, so rows stay 16-byte aligned
+    int64_t ldt_k = ldt;                         // leading dimension of the gathered operand in the kernel
     double* Bt = ws.get<double>((size_t)n * ldt);
     if (ws.failed) return SP_ERR_ALLOC;
     dim3 tg((unsigned)sp_ceil_div(n, 32), (unsigned)sp_ceil_div(K, 32));
@@ -156,8 +158,15 @@ extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const 
     const bool vec2 = (K % 2 == 0) && (lda % 2 == 0) && (reinterpret_cast<uintptr_t>(A) % 16 == 0) &&
                       (reinterpret_cast<uintptr_t>(Bt) % 16 == 0);
     const unsigned blocks = (unsigned)sp_ceil_div(part.nchunks * 32, kSThreads);
+    // The kernel keeps the operand row of the outer (segment) index in registers and gathers the
+    // row of the inner index: for column-major S the two operands simply trade places
+    // (segment = column j -> row j of B^T; inner coordinate = row i -> row i of A).
+    if (colmajor) {
+        const double* ta = A; A = Bt; Bt = const_cast<double*>(ta);
+        const int64_t tl = lda; lda = ldt; ldt_k = tl;
+    }
 #define SP_SDDMM_LAUNCH(V, NCH)                                                                                     \
-    k_sddmm<P, I, V, NCH><<<blocks, kSThreads, 0, stream>>>(pos, crd, S->val, outer, A, lda, Bt, ldt, K, x_vals,    \
+    k_sddmm<P, I, V, NCH><<<blocks, kSThreads, 0, stream>>>(pos, crd, S->val, outer, A, lda, Bt, ldt_k, K, x_vals,  \
                                                             part.row, part.nz, part.nchunks)
     SP_DISPATCH_WIDTHS(S, {
         const P* pos = static_cast<const P*>(S->pos[1]);

@@ -257,3 +257,44 @@ def test_every_kernel_with_wide_positions_and_coordinates(oracle, pb, cb, cbits)
             B5, C5 = I.dense_operand(3, 12, 96, R), I.dense_operand(3, 13, 96, R)
             r5, b5 = oracle.mttkrp(96, *t.coords, t.vals, B5, C5)
             assert_close(sp().sp_mttkrp(T, dev(B5), dev(C5)).cpu().numpy(), r5, b5, f"mttkrp R=5 widths {pb}/{cb}")
+
+
+@pytest.mark.parametrize("enc", ["CSC", "DCSC"])
+@pytest.mark.parametrize("K", [5, 64, 128, 300])
+def test_sddmm_column_major_sample(oracle, enc, K):
+    lt, od = MATRIX_ENCODINGS[enc]
+    for name, coo in [("uniform", I.uniform_matrix(300, 257, 4000, seed=1)), ("one_col", MATS[8][1]),
+                      ("powerlaw", I.config2(seed=2, n=900))]:
+        coords, vals = to_dev(coo)
+        S = sp().sp_pack(coo.dims, coords, vals, lt, od)
+        A = I.dense_operand(13, 8, coo.dims[0], K)
+        B = I.dense_operand(13, 9, K, coo.dims[1])
+        xg = sp().sp_sddmm(S, dev(A), dev(B)).cpu().numpy()
+        xe, be = oracle.sddmm(coo.coords[0], coo.coords[1], coo.vals, A, B)
+        ep = oracle.pack(coo.dims, coo.coords, coo.vals, lt, od).entry_pos
+        ref = np.empty_like(xe); bd = np.empty_like(be)
+        ref[ep] = xe; bd[ep] = be
+        assert_close(xg, ref, bd, f"sddmm {enc} {name} K={K}")
+
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("R", [5, 32])
+def test_mttkrp_any_output_mode(oracle, mode, R):
+    t = I.config5(seed=5, dim=150, nnz=30000)
+    dims = (150, 150, 150)
+    F = [I.dense_operand(6, 20 + d, 150, R) for d in range(3)]
+    others = [d for d in range(3) if d != mode]
+    # oracle: the mode-0 expression with the coordinates rotated so that `mode` comes first
+    ref, bd = oracle.mttkrp(dims[mode], t.coords[mode], t.coords[others[0]], t.coords[others[1]], t.vals,
+                            F[others[0]], F[others[1]])
+    coords, vals = to_dev(t)
+    for lt in [(1, 1, 1), (0, 1, 1)]:
+        for od in [(mode, others[0], others[1]), (mode, others[1], others[0])]:
+            T = sp().sp_pack(dims, coords, vals, lt, od)
+            M = sp().sp_mttkrp_mode(T, mode, [dev(f) for f in F]).cpu().numpy()
+            assert_close(M, ref, bd, f"mttkrp mode {mode} {lt} {od}")
+    b = sp()
+    Tbad = b.sp_pack(dims, coords, vals, (1, 1, 1), ((mode + 1) % 3, mode, 3 - mode - (mode + 1) % 3))
+    with pytest.raises(b.SpError) as e:
+        b.sp_mttkrp_mode(Tbad, mode, [dev(f) for f in F])
+    assert e.value.code == 2
