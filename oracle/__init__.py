@@ -162,3 +162,20 @@ def mttkrp(I, ti, tj, tk, tv, B, Cf, rows=None):
                           _ptr(M, _PD), _ptr(bd, _PD))
     assert rc == 0
     return M, bd
+
+
+def spmspm(m, kdim, n, ai, ak, av, bk, bj, bv):
+    """C = A * B, all sparse: returns CSR (pos, crd, val) of C and the per-entry bound sum|a*b|."""
+    ai, ak, av = _i64(ai), _i64(ak), _f64(av)
+    bk, bj, bv = _i64(bk), _i64(bj), _f64(bv)
+    f = lib().orc_spmspm
+    f.restype = C.c_int64
+    pos = np.zeros(m + 1, np.int64)
+    args = [C.c_int64(m), C.c_int64(kdim), C.c_int64(n), C.c_int64(av.size), _ptr(ai), _ptr(ak), _ptr(av, _PD),
+            C.c_int64(bv.size), _ptr(bk), _ptr(bj), _ptr(bv, _PD), _ptr(pos)]
+    total = f(*args, None, None, None)
+    assert total >= 0
+    crd = np.empty(total, np.int64); val = np.empty(total); bd = np.empty(total)
+    total2 = f(*args, _ptr(crd), _ptr(val, _PD), _ptr(bd, _PD))
+    assert total2 == total
+    return pos, crd, val, bd

@@ -268,3 +268,67 @@ int orc_mttkrp(int64_t nnz, const int64_t *ti, const int64_t *tj, const int64_t 
     free(acc); free(bnd);
     return 0;
 }
+
+/* ------------------------------------------------------------------------
+ * SpMSpM: C[i,j] = sum_k A[i,k] * B[k,j] with A, B and C all sparse (Section 4.3's
+ * kernel; Section 6.2, Table 2).  Inputs are coordinate lists; the result is returned
+ * row by row in increasing (i, j) order: every (i, j) for which some k has both
+ * A[i,k] and B[k,j] stored is an entry of C, even if its value cancels to zero.
+ * Pass 1 (crd_out == NULL) only counts; pass 2 fills.  Returns the entry count or -3.
+ * ---------------------------------------------------------------------- */
+static int cmp_i64(const void *a, const void *b)
+{
+    int64_t x = *(const int64_t *)a, y = *(const int64_t *)b;
+    return x < y ? -1 : (x > y ? 1 : 0);
+}
+
+int64_t orc_spmspm(int64_t m, int64_t kdim, int64_t n,
+                   int64_t annz, const int64_t *ai, const int64_t *ak, const double *av,
+                   int64_t bnnz, const int64_t *bk, const int64_t *bj, const double *bv,
+                   int64_t *pos_out /* m+1 */, int64_t *crd_out, double *val_out, double *bound_out)
+{
+    /* bucket the entries of A by row and of B by row (= k), keeping input order inside a bucket */
+    int64_t *astart = calloc((size_t)m + 2, sizeof(int64_t)), *bstart = calloc((size_t)kdim + 2, sizeof(int64_t));
+    int64_t *aord = malloc(sizeof(int64_t) * (size_t)(annz + 1)), *bord = malloc(sizeof(int64_t) * (size_t)(bnnz + 1));
+    long double *ws = calloc((size_t)n + 1, sizeof(long double)), *wb = calloc((size_t)n + 1, sizeof(long double));
+    char *mark = calloc((size_t)n + 1, 1);
+    int64_t *added = malloc(sizeof(int64_t) * (size_t)(n + 1));
+    if (!astart || !bstart || !aord || !bord || !ws || !wb || !mark || !added) return -3;
+    for (int64_t e = 0; e < annz; ++e) astart[ai[e] + 1]++;
+    for (int64_t e = 0; e < bnnz; ++e) bstart[bk[e] + 1]++;
+    for (int64_t r = 0; r < m; ++r) astart[r + 1] += astart[r];
+    for (int64_t r = 0; r < kdim; ++r) bstart[r + 1] += bstart[r];
+    {
+        int64_t *fill = calloc((size_t)(m > kdim ? m : kdim) + 1, sizeof(int64_t));
+        if (!fill) return -3;
+        for (int64_t e = 0; e < annz; ++e) aord[astart[ai[e]] + fill[ai[e]]++] = e;
+        memset(fill, 0, sizeof(int64_t) * (size_t)((m > kdim ? m : kdim) + 1));
+        for (int64_t e = 0; e < bnnz; ++e) bord[bstart[bk[e]] + fill[bk[e]]++] = e;
+        free(fill);
+    }
+    int64_t total = 0;
+    pos_out[0] = 0;
+    for (int64_t i = 0; i < m; ++i) {
+        int64_t count = 0;
+        for (int64_t p = astart[i]; p < astart[i + 1]; ++p) {
+            const int64_t ea = aord[p], k = ak[ea];
+            for (int64_t q = bstart[k]; q < bstart[k + 1]; ++q) {
+                const int64_t eb = bord[q], j = bj[eb];
+                const long double t = (long double)av[ea] * (long double)bv[eb];
+                if (!mark[j]) { mark[j] = 1; added[count++] = j; }     /* access pattern expansion */
+                ws[j] += t;
+                wb[j] += fabsl(t);
+            }
+        }
+        qsort(added, (size_t)count, sizeof(int64_t), cmp_i64);          /* insertion in index order */
+        for (int64_t c = 0; c < count; ++c) {
+            const int64_t j = added[c];
+            if (crd_out) { crd_out[total + c] = j; val_out[total + c] = (double)ws[j]; bound_out[total + c] = (double)wb[j]; }
+            ws[j] = 0; wb[j] = 0; mark[j] = 0;
+        }
+        total += count;
+        pos_out[i + 1] = total;
+    }
+    free(astart); free(bstart); free(aord); free(bord); free(ws); free(wb); free(mark); free(added);
+    return total;
+}

@@ -130,3 +130,37 @@ def test_extended_precision_accumulation(oracle):
     y, bd = oracle.spmv(1, rows, cols, v, np.ones(n))
     assert y[0] == 1.0 + 4096 * 2.0 ** -60 > 1.0
     assert bd[0] == y[0]
+
+
+@pytest.mark.parametrize("m,k,n,na,nb", [(9, 7, 8, 20, 25), (30, 30, 30, 90, 90), (5, 6, 4, 0, 10), (12, 3, 40, 36, 100)])
+def test_spmspm_matches_scipy_and_dense(oracle, m, k, n, na, nb):
+    A = I.uniform_matrix(m, k, na, seed=m)
+    B = I.uniform_matrix(k, n, nb, seed=n + 1)
+    pos, crd, val, bd = oracle.spmspm(m, k, n, A.coords[0], A.coords[1], A.vals, B.coords[0], B.coords[1], B.vals)
+    Ad, Bd = _dense(A), _dense(B)
+    # pattern: (i, j) is stored iff some k has A[i,k] and B[k,j] both stored
+    patt = ((Ad != 0).astype(np.int64) @ (Bd != 0).astype(np.int64)) > 0
+    got = np.zeros((m, n), bool)
+    rows = np.repeat(np.arange(m), np.diff(pos))
+    got[rows, crd] = True
+    assert np.array_equal(got, patt)
+    for i in range(m):
+        seg = crd[pos[i]:pos[i + 1]]
+        assert np.all(np.diff(seg) > 0)
+    ref = Ad @ Bd
+    refb = np.abs(Ad) @ np.abs(Bd)
+    assert _within(val, ref[rows, crd], refb[rows, crd])
+    assert np.allclose(bd, refb[rows, crd], rtol=1e-13, atol=0)
+    S = sp.csr_matrix(Ad) @ sp.csr_matrix(Bd)
+    S.sort_indices()
+    assert S.nnz <= crd.size           # scipy may drop nothing here, but never has more
+    assert np.allclose(S.toarray(), ref)
+
+
+def test_spmspm_result_density_matches_table_2(oracle):
+    # Section 6.2, Table 2: uniform random n x n operands of density 0.01 give rho_C = 0.10 at n = 1,024
+    n = 1024
+    A = I.uniform_matrix(n, n, int(0.01 * n * n), seed=21)
+    B = I.uniform_matrix(n, n, int(0.01 * n * n), seed=22)
+    pos, crd, val, bd = oracle.spmspm(n, n, n, A.coords[0], A.coords[1], A.vals, B.coords[0], B.coords[1], B.vals)
+    assert round(crd.size / (n * n), 2) == 0.10
