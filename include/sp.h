@@ -183,6 +183,21 @@ sp_status sp_mttkrp_mode(sp_tensor* T, int mode, const double* const* factors, i
                          double* M, void* stream);
 
 /*
+ * sp_spmspm - C[i,j] = sum_k A[i,k] * B[k,j] with all three matrices sparse and
+ * stored row-wise as (dense, compressed) with identity ordering - the SpMSpM
+ * kernel of Section 4.3 (access pattern expansion per row, insertion in index
+ * order), measured in Section 6.2.  A and B must share their bit widths;
+ * posBits / crdBits (0, 32, 64) are those of the result.  *out receives a new
+ * handle (release with sp_free) usable by every other call.  An (i,j) is stored
+ * in C when some k has both A[i,k] and B[k,j] stored, even if the sum cancels.
+ * Synchronises the stream once (the size of C depends on the data).  Sums are
+ * accumulated with floating-point atomics (order, and so the last bits, may
+ * vary from run to run).
+ */
+sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBits, int crdBits, void* stream,
+                    sp_tensor** out);
+
+/*
  * sp_spmv_static - y = A * x exactly as sp_spmv computes it (same kernels, same
  * results; the four encodings with a compressed inner level: CSR, DCSR, CSC, DCSC),
  * for callers that are not allowed to allocate device memory.

@@ -20,7 +20,7 @@ _LIB_PATH = os.path.join(_HERE, "libsp.so")
 
 SYMBOLS = ["sp_status_string", "sp_set_allocator", "sp_pack", "sp_free", "sp_info", "sp_positions",
            "sp_coordinates", "sp_values", "sp_unpack", "sp_spmv", "sp_spmm", "sp_sddmm", "sp_mttkrp",
-           "sp_set_profiling", "sp_get_pack_profile", "sp_launch_count", "sp_spmv_static", "sp_mttkrp_mode"]
+           "sp_set_profiling", "sp_get_pack_profile", "sp_launch_count", "sp_spmv_static", "sp_mttkrp_mode", "sp_spmspm"]
 SPMV_STATIC_MAX_ITEMS = 134217728
 
 
@@ -274,3 +274,11 @@ def sp_mttkrp_mode(T: SpTensor, mode: int, factors, M=None):
     ptrs = (C.c_void_p * 3)(*[f.data_ptr() if (f is not None and d != mode) else 0 for d, f in enumerate(factors)])
     _check(_lib.sp_mttkrp_mode(T._h, C.c_int(mode), ptrs, C.c_int64(R), _dptr(M), _stream()), "sp_mttkrp_mode")
     return M
+
+
+def sp_spmspm(A: SpTensor, B: SpTensor, posBits=32, crdBits=32) -> SpTensor:
+    """C = A * B with A, B, C all CSR; returns a new handle."""
+    use_torch_allocator()
+    h = C.c_void_p()
+    _check(_lib.sp_spmspm(A._h, B._h, C.c_int(posBits), C.c_int(crdBits), _stream(), C.byref(h)), "sp_spmspm")
+    return SpTensor(h)
