@@ -60,6 +60,9 @@ def make_workload(small: bool, seed: int):
     wl["B4"] = I.dense_operand(seed, 36, 128, c4.dims[1])
     wl["Bf"] = I.dense_operand(seed, 37, c5.dims[1], 32)
     wl["Cf"] = I.dense_operand(seed, 38, c5.dims[2], 32)
+    nq = 1024 if small else 8192      # SpMSpM (a "next" row, timed on its own, not part of the step): Table 2's largest shape
+    wl["q_a"] = I.uniform_matrix(nq, nq, int(0.01 * nq * nq), seed + 41)
+    wl["q_b"] = I.uniform_matrix(nq, nq, int(0.01 * nq * nq), seed + 42)
     return wl
 
 
@@ -114,6 +117,8 @@ class GpuSuite:
         self.A1c = sp.sp_pack(wl["c1b"].dims, i32(wl["c1b"]), dev(wl["c1b"].vals), (1, 0))
         self.S4 = sp.sp_pack(wl["c4"].dims, i32(wl["c4"]), dev(wl["c4"].vals), (0, 1))
         self.xv4 = f64(self.S4.nval)
+        self.Qa = sp.sp_pack(wl["q_a"].dims, i32(wl["q_a"]), dev(wl["q_a"].vals), (0, 1))
+        self.Qb = sp.sp_pack(wl["q_b"].dims, i32(wl["q_b"]), dev(wl["q_b"].vals), (0, 1))
         self.flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
         torch.cuda.synchronize()
 
@@ -160,6 +165,7 @@ class GpuSuite:
             "sddmm_csr": lambda: sp.sp_sddmm(self.S4, self.A4, self.B4, self.xv4),
             "pack_csf": lambda: sp.sp_pack(wl["c5"].dims, self.c5, self.v5, (1, 1, 1)).free(),
             "mttkrp_csf": lambda: sp.sp_mttkrp(csf(), self.Bf, self.Cf, self.M5),
+            "next_spmspm_csr": lambda: sp.sp_spmspm(self.Qa, self.Qb).free(),
         }
 
     def flush_l2(self):
@@ -390,6 +396,13 @@ def main():
     # ---- each call on its own (rank 0 only decides the report; all ranks run it to stay in step)
     kernels = {}
     calls = suite.calls()
+    qa, qb = wl["q_a"], wl["q_b"]
+    rowlen_b = np.bincount(qb.coords[0], minlength=qb.dims[0])
+    products = int(rowlen_b[qa.coords[1]].sum())
+    qc = sp.sp_spmspm(suite.Qa, suite.Qb)
+    model["next_spmspm_csr"] = dict(flops=2 * products, bytes=12 * (qa.nnz + qb.nnz + qc.nval) + 4 * 3 * (qa.dims[0] + 1),
+                                    units=products)
+    qc.free()
     for name, fn in calls.items():
         ts = suite.time_call(fn, args.kernel_reps)
         med = statistics.median(ts)

@@ -148,9 +148,8 @@ def test_unsupported_encodings():
     with pytest.raises(b.SpError) as e:
         b.sp_spmv(T, dev(np.ones(20)))
     assert e.value.code == 2
-    S = b.sp_pack(coo.dims, coords, vals, (0, 1), (1, 0))
-    with pytest.raises(b.SpError) as e:
-        b.sp_sddmm(S, dev(np.ones((20, 4))), dev(np.ones((4, 20))))
+    with pytest.raises(b.SpError) as e:          # MTTKRP wants a rank-3 tensor
+        b.sp_mttkrp(b.sp_pack(coo.dims, coords, vals, (0, 1)), dev(np.ones((20, 4))), dev(np.ones((20, 4))))
     assert e.value.code == 2
 
 
