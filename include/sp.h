@@ -130,6 +130,16 @@ sp_status sp_unpack(const sp_tensor* t, void* const* coo_coords_out, double* val
                     int64_t* nnz_out, void* stream);
 
 /*
+ * sp_convert - re-encode a tensor (the convert operation of Section 4.2, which
+ * the paper implements through an intermediate coordinate scheme, as here:
+ * sp_unpack followed by sp_pack, all on the device).  Every stored value of the
+ * source, explicit zeros included, becomes a stored entry of the result.
+ * Synchronises the stream as sp_pack does.  *out: a new handle.
+ */
+sp_status sp_convert(const sp_tensor* t, const sp_level_type* dimLevelType, const int* dimOrdering,
+                     int posBits, int crdBits, void* stream, sp_tensor** out);
+
+/*
  * sp_spmv - y[i] = sum_k A[i,k] * x[k]  (the matvec of Section 6.2).
  * A: rank 2, any of the eight encodings: level types (dense, compressed) or
  * (compressed, compressed) in either ordering (CSR, DCSR, CSC, DCSC), and

@@ -20,7 +20,7 @@ _LIB_PATH = os.path.join(_HERE, "libsp.so")
 
 SYMBOLS = ["sp_status_string", "sp_set_allocator", "sp_pack", "sp_free", "sp_info", "sp_positions",
            "sp_coordinates", "sp_values", "sp_unpack", "sp_spmv", "sp_spmm", "sp_sddmm", "sp_mttkrp",
-           "sp_set_profiling", "sp_get_pack_profile", "sp_launch_count", "sp_spmv_static", "sp_mttkrp_mode", "sp_spmspm"]
+           "sp_set_profiling", "sp_get_pack_profile", "sp_launch_count", "sp_spmv_static", "sp_mttkrp_mode", "sp_spmspm", "sp_convert"]
 SPMV_STATIC_MAX_ITEMS = 134217728
 
 
@@ -281,4 +281,14 @@ def sp_spmspm(A: SpTensor, B: SpTensor, posBits=32, crdBits=32) -> SpTensor:
     use_torch_allocator()
     h = C.c_void_p()
     _check(_lib.sp_spmspm(A._h, B._h, C.c_int(posBits), C.c_int(crdBits), _stream(), C.byref(h)), "sp_spmspm")
+    return SpTensor(h)
+
+
+def sp_convert(t: SpTensor, dimLevelType, dimOrdering=None, posBits=32, crdBits=32) -> SpTensor:
+    """Re-encode a tensor through coordinates (unpack + pack on the device)."""
+    use_torch_allocator()
+    h = C.c_void_p()
+    lt = (C.c_int * t.rank)(*[int(x) for x in dimLevelType])
+    od = (C.c_int * t.rank)(*[int(o) for o in dimOrdering]) if dimOrdering is not None else None
+    _check(_lib.sp_convert(t._h, lt, od, C.c_int(posBits), C.c_int(crdBits), _stream(), C.byref(h)), "sp_convert")
     return SpTensor(h)

@@ -846,3 +846,24 @@ extern "C" sp_status sp_unpack(const sp_tensor* t, void* const* coo_coords_out, 
     }
     return SP_OK;
 }
+
+// sp_convert: storage -> coordinates -> storage (Section 4.2: conversions between sparse formats go
+// through an intermediate coordinate scheme rather than one direct converter per pair of formats).
+extern "C" sp_status sp_convert(const sp_tensor* t, const sp_level_type* dimLevelType, const int* dimOrdering,
+                                int posBits, int crdBits, void* stream_, sp_tensor** out) {
+    if (!out) return SP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!t || !dimLevelType) return SP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    sp_workspace ws(stream);
+    const int64_t n = t->nval;
+    void* coords[SP_MAX_RANK] = {};
+    for (int d = 0; d < t->rank; ++d) coords[d] = ws.get<int64_t>((size_t)n);
+    double* vals = ws.get<double>((size_t)n);
+    if (ws.failed) return SP_ERR_ALLOC;
+    int64_t cnt = 0;
+    sp_status st = sp_unpack(t, coords, vals, &cnt, stream_);
+    if (st != SP_OK) return st;
+    return sp_pack(t->rank, t->dims, cnt, coords, 64, vals, dimLevelType, dimOrdering, posBits, crdBits, SP_DUP_SUM,
+                   stream_, out);
+}

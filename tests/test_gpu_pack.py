@@ -176,3 +176,25 @@ def test_all_compressed_four_and_five_dimensional_shapes(oracle, dims, nnz):
     od = tuple(reversed(range(len(dims))))
     t = sp().sp_pack(dims, coords, vals, lt, od)
     assert_storage_equal(t, oracle.pack(dims, coo.coords, coo.vals, lt, od))
+
+
+def test_convert_between_encodings(oracle):
+    # Section 4.2's example converts CSR to CSC; every pair of all-compressed / CSR-like encodings here
+    coo = I.uniform_matrix(60, 45, 700, seed=9)
+    coords, vals = to_dev(coo)
+    encs = [((0, 1), (0, 1)), ((0, 1), (1, 0)), ((1, 1), (0, 1)), ((1, 1), (1, 0))]
+    for lt_a, od_a in encs:
+        src = sp().sp_pack(coo.dims, coords, vals, lt_a, od_a)
+        for lt_b, od_b in encs:
+            dst = sp().sp_convert(src, lt_b, od_b, 64, 32)
+            assert_storage_equal(dst, oracle.pack(coo.dims, coo.coords, coo.vals, lt_b, od_b))
+    t3 = I.uniform_tensor((9, 8, 7), 200, seed=10)
+    c3, v3 = to_dev(t3)
+    src = sp().sp_pack(t3.dims, c3, v3, (1, 1, 1))
+    dst = sp().sp_convert(src, (0, 1, 1), (0, 2, 1))
+    assert_storage_equal(dst, oracle.pack(t3.dims, t3.coords, t3.vals, (0, 1, 1), (0, 2, 1)))
+    # from a dense-inner encoding the explicit zeros travel along as stored entries
+    cdr = sp().sp_pack(coo.dims, coords, vals, (1, 0))
+    back = sp().sp_convert(cdr, (0, 1))
+    oc, ov = oracle.unpack(oracle.pack(coo.dims, coo.coords, coo.vals, (1, 0)))
+    assert_storage_equal(back, oracle.pack(coo.dims, oc, ov, (0, 1)))
