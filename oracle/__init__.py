@@ -179,3 +179,13 @@ def spmspm(m, kdim, n, ai, ak, av, bk, bj, bv):
     total2 = f(*args, _ptr(crd), _ptr(val, _PD), _ptr(bd, _PD))
     assert total2 == total
     return pos, crd, val, bd
+
+
+def vec_dot(ai, av, bi, bv):
+    """Inner product of two sparse vectors given as sorted (coordinates, values); returns (x, bound)."""
+    ai, av, bi, bv = _i64(ai), _f64(av), _i64(bi), _f64(bv)
+    f = lib().orc_vec_dot
+    f.restype = C.c_double
+    bd = C.c_double()
+    x = f(C.c_int64(av.size), _ptr(ai), _ptr(av, _PD), C.c_int64(bv.size), _ptr(bi), _ptr(bv, _PD), C.byref(bd))
+    return float(x), float(bd.value)

@@ -332,3 +332,29 @@ int64_t orc_spmspm(int64_t m, int64_t kdim, int64_t n,
     free(astart); free(bstart); free(aord); free(bord); free(ws); free(wb); free(mark); free(added);
     return total;
 }
+
+/* ------------------------------------------------------------------------
+ * Sparse-sparse inner product x = sum_i a[i] * b[i] of two compressed vectors, by the
+ * co-iteration of Section 4.3: both coordinate lists (sorted, as storage keeps them) are
+ * walked together, the smaller index advances, and a product is formed only where the two
+ * indices meet.  Returns the f64 rounding of the extended-precision sum; *bound = sum|a*b|.
+ * ---------------------------------------------------------------------- */
+double orc_vec_dot(int64_t na, const int64_t *ai, const double *av, int64_t nb, const int64_t *bi, const double *bv,
+                   double *bound)
+{
+    long double acc = 0.0L, bnd = 0.0L;
+    int64_t ia = 0, ib = 0;
+    while (ia < na && ib < nb) {
+        const int64_t ixa = ai[ia], ixb = bi[ib];
+        const int64_t i = ixa < ixb ? ixa : ixb;
+        if (ixa == i && ixb == i) {
+            const long double t = (long double)av[ia] * (long double)bv[ib];
+            acc += t;
+            bnd += fabsl(t);
+        }
+        if (ixa == i) ++ia;
+        if (ixb == i) ++ib;
+    }
+    if (bound) *bound = (double)bnd;
+    return (double)acc;
+}

@@ -164,3 +164,16 @@ def test_spmspm_result_density_matches_table_2(oracle):
     B = I.uniform_matrix(n, n, int(0.01 * n * n), seed=22)
     pos, crd, val, bd = oracle.spmspm(n, n, n, A.coords[0], A.coords[1], A.vals, B.coords[0], B.coords[1], B.vals)
     assert round(crd.size / (n * n), 2) == 0.10
+
+
+@pytest.mark.parametrize("n,na,nb", [(50, 10, 12), (1000, 300, 400), (20, 0, 5), (64, 64, 64)])
+def test_sparse_dot_by_co_iteration(oracle, n, na, nb):
+    a = I.uniform_tensor((n,), na, seed=n)
+    b = I.uniform_tensor((n,), nb, seed=n + 7)
+    oa, ob = np.argsort(a.coords[0]), np.argsort(b.coords[0])
+    x, bd = oracle.vec_dot(a.coords[0][oa], a.vals[oa], b.coords[0][ob], b.vals[ob])
+    da, db = np.zeros(n), np.zeros(n)
+    da[a.coords[0]] = a.vals; db[b.coords[0]] = b.vals
+    assert abs(x - float(da @ db)) <= 1e-12 * float(np.abs(da) @ np.abs(db)) + 0.0
+    assert np.isclose(bd, float(np.abs(da) @ np.abs(db)), rtol=1e-13, atol=0)
+    assert oracle.vec_dot(a.coords[0][oa], a.vals[oa], a.coords[0][oa], np.ones(na))[0] == pytest.approx(a.vals.sum(), abs=1e-12)
