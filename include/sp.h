@@ -193,6 +193,21 @@ sp_status sp_mttkrp_mode(sp_tensor* T, int mode, const double* const* factors, i
                          double* M, void* stream);
 
 /*
+ * sp_scale - x[..] *= c over the stored values only, in place (Section 4.3's first example:
+ * the loop body runs only for stored entries).  Any rank and encoding.  This is the one call
+ * that changes a handle's values; cached work partitions stay valid (structure is untouched).
+ */
+sp_status sp_scale(sp_tensor* x, double c, void* stream);
+
+/*
+ * sp_vec_dot - *result = sum_i a[i] * b[i] for two compressed vectors (rank 1, level type
+ * compressed) of equal length and equal coordinate width: the co-iteration example of
+ * Section 4.3 (a product only where both store the index).  result: device, one double.
+ * Partial sums are combined with atomic adds.
+ */
+sp_status sp_vec_dot(const sp_tensor* a, const sp_tensor* b, double* result, void* stream);
+
+/*
  * sp_spmspm - C[i,j] = sum_k A[i,k] * B[k,j] with all three matrices sparse and
  * stored row-wise as (dense, compressed) with identity ordering - the SpMSpM
  * kernel of Section 4.3 (access pattern expansion per row, insertion in index

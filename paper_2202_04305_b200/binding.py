@@ -20,7 +20,7 @@ _LIB_PATH = os.path.join(_HERE, "libsp.so")
 
 SYMBOLS = ["sp_status_string", "sp_set_allocator", "sp_pack", "sp_free", "sp_info", "sp_positions",
            "sp_coordinates", "sp_values", "sp_unpack", "sp_spmv", "sp_spmm", "sp_sddmm", "sp_mttkrp",
-           "sp_set_profiling", "sp_get_pack_profile", "sp_launch_count", "sp_spmv_static", "sp_mttkrp_mode", "sp_spmspm", "sp_convert"]
+           "sp_set_profiling", "sp_get_pack_profile", "sp_launch_count", "sp_spmv_static", "sp_mttkrp_mode", "sp_spmspm", "sp_convert", "sp_scale", "sp_vec_dot"]
 SPMV_STATIC_MAX_ITEMS = 134217728
 
 
@@ -292,3 +292,14 @@ def sp_convert(t: SpTensor, dimLevelType, dimOrdering=None, posBits=32, crdBits=
     od = (C.c_int * t.rank)(*[int(o) for o in dimOrdering]) if dimOrdering is not None else None
     _check(_lib.sp_convert(t._h, lt, od, C.c_int(posBits), C.c_int(crdBits), _stream(), C.byref(h)), "sp_convert")
     return SpTensor(h)
+
+
+def sp_scale(x: SpTensor, c: float):
+    _check(_lib.sp_scale(x._h, C.c_double(c), _stream()), "sp_scale")
+    return x
+
+
+def sp_vec_dot(a: SpTensor, b: SpTensor):
+    out = torch.empty(1, dtype=torch.float64, device="cuda")
+    _check(_lib.sp_vec_dot(a._h, b._h, _dptr(out), _stream()), "sp_vec_dot")
+    return out
