@@ -88,7 +88,13 @@ sp_status sp_set_allocator(void* (*alloc)(size_t bytes, void* stream, void* ctx)
  *   coo_vals        device, nnz doubles
  *   dimLevelType    host, per level
  *   dimOrdering     host, per level: logical dimension stored at level l; NULL = identity
- *   posBits/crdBits 0 (= 64, the "native" width), 32 or 64; stored unsigned
+ *   posBits/crdBits 0 (= 64, the "native" width), 8, 16, 32 or 64 (Section 4.1); stored
+ *                   unsigned.  A width too small for the largest position (the entry
+ *                   count of a level) or for a compressed level's largest possible
+ *                   coordinate (its size - 1) yields SP_ERR_WIDTH_OVERFLOW.  The compute
+ *                   kernels read 8- and 16-bit arrays through a 32-bit copy that the
+ *                   handle builds (through the allocator) on the first such call and
+ *                   keeps until sp_free; the accessors always return the narrow arrays.
  *   flags           SP_DUP_SUM or SP_DUP_ERROR
  *   out             receives the handle; release with sp_free
  *
@@ -212,7 +218,7 @@ sp_status sp_vec_dot(const sp_tensor* a, const sp_tensor* b, double* result, voi
  * stored row-wise as (dense, compressed) with identity ordering - the SpMSpM
  * kernel of Section 4.3 (access pattern expansion per row, insertion in index
  * order), measured in Section 6.2.  A and B must share their bit widths;
- * posBits / crdBits (0, 32, 64) are those of the result.  *out receives a new
+ * posBits / crdBits (0, 8, 16, 32, 64) are those of the result.  *out receives a new
  * handle (release with sp_free) usable by every other call.  An (i,j) is stored
  * in C when some k has both A[i,k] and B[k,j] stored, even if the sum cancels.
  * Synchronises the stream once (the size of C depends on the data).  Sums are
@@ -239,6 +245,8 @@ sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBits, int crd
  *
  * Its scratch is a fixed array compiled into the library (about 2 MiB of device
  * memory on every GPU that loads the library, held until the process exits).
+ * Handles with 8- or 16-bit arrays are refused with SP_ERR_UNSUPPORTED (reading
+ * them would need the allocated 32-bit copy).
  * Capacity: rows-or-columns stored at the compressed level plus stored entries,
  * i.e. (sp_positions(A, 1) len - 1) + (sp_coordinates(A, 1) len), must not exceed
  * SP_SPMV_STATIC_MAX_ITEMS; larger inputs are refused with SP_ERR_TOO_LARGE and

@@ -89,6 +89,16 @@ def pack(dims, coords, vals, lt, ord=None) -> Storage:
     return Storage(tuple(int(d) for d in dims), tuple(int(t) for t in lt), ord, pos, crd, val, ep)
 
 
+def min_widths(s: Storage):
+    """Section 4.1's rule on pointerBitWidth / indexBitWidth: a width is usable when the largest stored
+    position (resp. coordinate) fits it.  Returns the smallest admissible (position, coordinate) widths
+    among 8, 16, 32, 64; the coordinate bound is the level size, not the largest coordinate present."""
+    pmax = max([int(p.max()) for p in s.pos if p is not None and p.size] + [0])
+    cmax = max([int(s.dims[s.ord[l]]) - 1 for l in range(len(s.dims)) if s.lt[l] == COMPRESSED] + [0])
+    fit = lambda v: next(w for w in (8, 16, 32, 64) if v < (1 << w))
+    return fit(pmax), fit(cmax)
+
+
 def unpack(s: Storage):
     """Stored entries in storage order as (logical coords per dim, values)."""
     rank = len(s.dims)

@@ -101,6 +101,9 @@ class _DevArray:
         self._owner = owner
 
 
+_WIDTH_VIEW = {8: (torch.uint8, "|u1"), 16: (torch.uint16, "<u2"), 32: (torch.int32, "<i4"), 64: (torch.int64, "<i8")}
+
+
 class SpTensor:
     """Owner of an sp_tensor handle."""
 
@@ -121,13 +124,14 @@ class SpTensor:
     def _arr(self, fn, level, bits):
         p, n = C.c_void_p(), C.c_int64()
         _check(fn(self._h, C.c_int(level), C.byref(p), C.byref(n)), fn.__name__)
-        dt = torch.int32 if bits == 32 else torch.int64
+        dt, typestr = _WIDTH_VIEW[bits]
         if n.value == 0 or not p.value:
             return torch.empty(0, dtype=dt, device="cuda")
-        return torch.as_tensor(_DevArray(p.value, n.value, "<i4" if bits == 32 else "<i8", self), device="cuda")
+        return torch.as_tensor(_DevArray(p.value, n.value, typestr, self), device="cuda")
 
     def positions(self, level):
-        """pos[level] as a signed view of the unsigned device array (empty at dense levels)."""
+        """pos[level] as a view of the device array (empty at dense levels): uint8 / uint16 for the
+        narrow widths, a signed view of the unsigned words for 32 and 64 bits."""
         return self._arr(_lib.sp_positions, level, self.pos_bits)
 
     def coordinates(self, level):

@@ -62,7 +62,8 @@ sp_status sp_free(sp_tensor* t) {
         sp_dev_free(t->pos[l], nullptr);
         sp_dev_free(t->crd[l], nullptr);
     }
-    sp_dev_free(t->val, nullptr);
+    if (t->owns_val) sp_dev_free(t->val, nullptr);
+    if (t->wide) sp_free(t->wide);
     for (auto& kv : t->parts) {
         sp_dev_free(kv.second.row, nullptr);
         sp_dev_free(kv.second.nz, nullptr);

@@ -40,7 +40,16 @@ struct sp_tensor {
     int device = 0;
     std::mutex mu;
     std::map<uint64_t, sp_partition> parts;   // key = (kind << 32) | items per chunk
+    // For handles stored with 8- or 16-bit positions/coordinates: a copy of the overhead arrays
+    // widened to 32 bits that the compute kernels read (values shared, not copied).  Built on
+    // first use by sp_widened(), owned by this handle.
+    sp_tensor* wide = nullptr;
+    bool owns_val = true;
 };
+
+// The handle the compute kernels should read: t itself when its widths are 32 or 64 bits,
+// otherwise its (cached) 32-bit shadow.
+sp_status sp_widened(sp_tensor* t, cudaStream_t stream, sp_tensor** out);
 
 // ---------------------------------------------------------------------------
 // Allocation through the installed allocator
@@ -81,18 +90,30 @@ void sp_count_launches(int n);
 #define SP_LAUNCH_CHECK() SP_CUDA(cudaGetLastError())
 
 static inline int64_t sp_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+static inline bool sp_valid_width(int bits) { return bits == 8 || bits == 16 || bits == 32 || bits == 64; }
+static inline uint64_t sp_width_max(int bits) { return bits >= 64 ? ~0ull : ((1ull << bits) - 1ull); }
 
 // ---------------------------------------------------------------------------
 // Device helpers
 // ---------------------------------------------------------------------------
 #ifdef __CUDACC__
 
-__device__ __forceinline__ uint64_t sp_load_uint(const void* base, int64_t i, bool is64) {
-    return is64 ? static_cast<const uint64_t*>(base)[i] : static_cast<const uint32_t*>(base)[i];
+// Element i of an unsigned array whose element width (8, 16, 32 or 64 bits) is known at run time.
+__device__ __forceinline__ uint64_t sp_load_uint(const void* base, int64_t i, int bits) {
+    switch (bits) {
+        case 64: return static_cast<const uint64_t*>(base)[i];
+        case 32: return static_cast<const uint32_t*>(base)[i];
+        case 16: return static_cast<const uint16_t*>(base)[i];
+        default: return static_cast<const uint8_t*>(base)[i];
+    }
 }
-__device__ __forceinline__ void sp_store_uint(void* base, int64_t i, uint64_t v, bool is64) {
-    if (is64) static_cast<uint64_t*>(base)[i] = v;
-    else static_cast<uint32_t*>(base)[i] = static_cast<uint32_t>(v);
+__device__ __forceinline__ void sp_store_uint(void* base, int64_t i, uint64_t v, int bits) {
+    switch (bits) {
+        case 64: static_cast<uint64_t*>(base)[i] = v; break;
+        case 32: static_cast<uint32_t*>(base)[i] = static_cast<uint32_t>(v); break;
+        case 16: static_cast<uint16_t*>(base)[i] = static_cast<uint16_t>(v); break;
+        default: static_cast<uint8_t*>(base)[i] = static_cast<uint8_t>(v); break;
+    }
 }
 
 __device__ __forceinline__ unsigned sp_lane() { return threadIdx.x & 31u; }

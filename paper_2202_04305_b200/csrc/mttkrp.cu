@@ -408,6 +408,12 @@ extern "C" sp_status sp_mttkrp_mode(sp_tensor* T, int mode, const double* const*
 }
 
 static sp_status mttkrp_levels(sp_tensor* T, const double* F1, const double* F2, int64_t R, double* M, cudaStream_t stream) {
+    {   // 8- and 16-bit storage is read through its 32-bit shadow
+        sp_tensor* wide_ = nullptr;
+        const sp_status ws_ = sp_widened(T, stream, &wide_);
+        if (ws_ != SP_OK) return ws_;
+        T = wide_;
+    }
     const double* B = F1;
     const double* C = F2;
     SP_CUDA(cudaMemsetAsync(M, 0, (size_t)T->dims[T->ord[0]] * R * sizeof(double), stream));

@@ -373,7 +373,7 @@ struct EmitArgs {
     void* crd[SP_MAX_RANK];
     double* val;
     uint32_t* seg_out;   // optional: level-0 coordinate of every stored entry (column-major matrices)
-    bool pos64, crd64;
+    int posBits, crdBits;
     unsigned flags;
     int* err;
 };
@@ -437,8 +437,8 @@ __global__ void __launch_bounds__(kCtThreads) k_emit(EmitArgs a) {
             } else {
                 const int64_t nid = incl[l] - 1;
                 if (fl) {
-                    sp_store_uint(a.crd[l], nid, (uint64_t)c, a.crd64);
-                    if (e == 0 || pprev != ppos) sp_store_uint(a.pos[l], ppos, (uint64_t)nid, a.pos64);
+                    sp_store_uint(a.crd[l], nid, (uint64_t)c, a.crdBits);
+                    if (e == 0 || pprev != ppos) sp_store_uint(a.pos[l], ppos, (uint64_t)nid, a.posBits);
                 }
                 pprev = nid - (fl ? 1 : 0);
                 ppos = nid;
@@ -460,7 +460,7 @@ __global__ void __launch_bounds__(kCtThreads) k_emit(EmitArgs a) {
     }
 }
 
-__global__ void k_store_one(void* base, int64_t i, uint64_t v, bool is64) { sp_store_uint(base, i, v, is64); }
+__global__ void k_store_one(void* base, int64_t i, uint64_t v, int bits) { sp_store_uint(base, i, v, bits); }
 
 // --------------------------------------------- suffix-min fill of pos[] ---
 // a[i] <- min(a[i..L-1]).  Written as a forward scan over r = L-1-i.
@@ -570,7 +570,7 @@ struct UnpackArgs {
     const void* crd[SP_MAX_RANK];
     const double* val;
     int64_t nval;
-    bool pos64, crd64;
+    int posBits, crdBits;
     int64_t* out[SP_MAX_RANK];
     double* vals_out;
 };
@@ -586,12 +586,12 @@ __global__ void k_unpack(UnpackArgs a) {
             c = p % a.sz[l];
             p /= a.sz[l];
         } else {
-            c = (int64_t)sp_load_uint(a.crd[l], p, a.crd64);
+            c = (int64_t)sp_load_uint(a.crd[l], p, a.crdBits);
             // parent = last index whose offset is <= p
             int64_t lo = 0, hi = a.npos[l] - 1;   // answer in [0, npos-2]
             while (hi - lo > 1) {
                 int64_t mid = (lo + hi) >> 1;
-                if ((int64_t)sp_load_uint(a.pos[l], mid, a.pos64) <= p) lo = mid; else hi = mid;
+                if ((int64_t)sp_load_uint(a.pos[l], mid, a.posBits) <= p) lo = mid; else hi = mid;
             }
             p = lo;
         }
@@ -619,7 +619,7 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
     if (coo_coord_bits != 32 && coo_coord_bits != 64) return SP_ERR_INVALID_ARG;
     if (posBits == 0) posBits = 64;
     if (crdBits == 0) crdBits = 64;
-    if ((posBits != 32 && posBits != 64) || (crdBits != 32 && crdBits != 64)) return SP_ERR_INVALID_ARG;
+    if (!sp_valid_width(posBits) || !sp_valid_width(crdBits)) return SP_ERR_INVALID_ARG;
     if (flags > SP_DUP_ERROR) return SP_ERR_INVALID_ARG;
     if (nnz >= ((int64_t)1 << 32)) return SP_ERR_UNSUPPORTED;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -645,8 +645,8 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
     if (total_bits > 63) return SP_ERR_UNSUPPORTED;
     for (int l = 0, s = total_bits; l < rank; ++l) { s -= plan.bits[l]; plan.shift[l] = s; }
 
-    const uint64_t max_pos = posBits == 32 ? 0xffffffffull : ~0ull;
-    const uint64_t max_crd = crdBits == 32 ? 0xffffffffull : ~0ull;
+    const uint64_t max_pos = sp_width_max(posBits);
+    const uint64_t max_crd = sp_width_max(crdBits);
     for (int l = 0; l < rank; ++l)
         if (plan.lt[l] == SP_COMPRESSED && (uint64_t)(plan.sz[l] - 1) > max_crd) return SP_ERR_WIDTH_OVERFLOW;
 
@@ -771,7 +771,7 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
         a.keys = keys; a.idx = idx; a.vals_in = coo_vals; a.n = n; a.plan = plan;
         a.tileprefix = tileprefix; a.ntiles = ct_tiles;
         for (int l = 0; l < SP_MAX_RANK; ++l) { a.pos[l] = t->pos[l]; a.crd[l] = t->crd[l]; }
-        a.val = t->val; a.pos64 = posBits == 64; a.crd64 = crdBits == 64; a.flags = flags; a.err = d_err;
+        a.val = t->val; a.posBits = posBits; a.crdBits = crdBits; a.flags = flags; a.err = d_err;
         // Column-major matrices run SpMM as a flat loop over entries and need each entry's column:
         // it is in the sorted key anyway, so it is written here instead of being searched for later.
         a.seg_out = nullptr;
@@ -786,11 +786,13 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
         sp_count_launches(1);
         for (int l = 0; l < rank; ++l) {
             if (plan.lt[l] != SP_COMPRESSED) continue;
-            k_store_one<<<1, 1, 0, stream>>>(t->pos[l], parents_at[l], (uint64_t)counts[l], posBits == 64);
+            k_store_one<<<1, 1, 0, stream>>>(t->pos[l], parents_at[l], (uint64_t)counts[l], posBits);
             sp_count_launches(1);
             if (needs_fill[l]) {
-                sp_status s2 = posBits == 64 ? suffix_min_inplace<uint64_t>(t->pos[l], t->npos[l], stream)
-                                             : suffix_min_inplace<uint32_t>(t->pos[l], t->npos[l], stream);
+                sp_status s2 = posBits == 64   ? suffix_min_inplace<uint64_t>(t->pos[l], t->npos[l], stream)
+                               : posBits == 32 ? suffix_min_inplace<uint32_t>(t->pos[l], t->npos[l], stream)
+                               : posBits == 16 ? suffix_min_inplace<uint16_t>(t->pos[l], t->npos[l], stream)
+                                               : suffix_min_inplace<uint8_t>(t->pos[l], t->npos[l], stream);
                 if (s2 != SP_OK) return fail(s2);
             }
         }
@@ -835,8 +837,8 @@ extern "C" sp_status sp_unpack(const sp_tensor* t, void* const* coo_coords_out, 
     }
     a.val = t->val;
     a.nval = t->nval;
-    a.pos64 = t->posBits == 64;
-    a.crd64 = t->crdBits == 64;
+    a.posBits = t->posBits;
+    a.crdBits = t->crdBits;
     a.vals_out = vals_out;
     *nnz_out = t->nval;
     if (t->nval > 0) {

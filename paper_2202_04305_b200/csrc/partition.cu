@@ -123,6 +123,61 @@ sp_status sp_get_merge_partition(sp_tensor* t, int64_t items, int64_t carry_elem
     return SP_OK;
 }
 
+// ------------------------------------------------------------------ widened shadow ---
+namespace {
+template <typename S>
+__global__ void k_widen(const S* __restrict__ src, uint32_t* __restrict__ dst, int64_t n) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        dst[i] = (uint32_t)src[i];
+}
+
+// A 32-bit (or, for bits >= 32, plain) copy of an overhead array.
+sp_status widen_array(const void* src, int64_t n, int bits, cudaStream_t stream, void** out) {
+    *out = nullptr;
+    if (!src) return SP_OK;
+    const int obits = bits < 32 ? 32 : bits;
+    void* d = sp_dev_alloc((size_t)(n ? n : 1) * (obits / 8), stream);
+    if (!d) return SP_ERR_ALLOC;
+    *out = d;
+    if (n == 0) return SP_OK;
+    if (bits >= 32) {
+        SP_CUDA(cudaMemcpyAsync(d, src, (size_t)n * (bits / 8), cudaMemcpyDeviceToDevice, stream));
+        return SP_OK;
+    }
+    const unsigned blocks = (unsigned)std::min<int64_t>(sp_ceil_div(n, 256), 148 * 8);
+    if (bits == 16) k_widen<uint16_t><<<blocks, 256, 0, stream>>>(static_cast<const uint16_t*>(src), static_cast<uint32_t*>(d), n);
+    else k_widen<uint8_t><<<blocks, 256, 0, stream>>>(static_cast<const uint8_t*>(src), static_cast<uint32_t*>(d), n);
+    SP_LAUNCH_CHECK();
+    sp_count_launches(1);
+    return SP_OK;
+}
+}  // namespace
+
+sp_status sp_widened(sp_tensor* t, cudaStream_t stream, sp_tensor** out) {
+    if (t->posBits >= 32 && t->crdBits >= 32) { *out = t; return SP_OK; }
+    std::lock_guard<std::mutex> lock(t->mu);
+    if (t->wide) { *out = t->wide; return SP_OK; }
+    sp_tensor* w = new sp_tensor();
+    w->rank = t->rank;
+    w->device = t->device;
+    w->posBits = t->posBits < 32 ? 32 : t->posBits;
+    w->crdBits = t->crdBits < 32 ? 32 : t->crdBits;
+    w->val = t->val;
+    w->nval = t->nval;
+    w->owns_val = false;
+    sp_status st = SP_OK;
+    for (int l = 0; l < t->rank; ++l) {
+        w->dims[l] = t->dims[l]; w->lt[l] = t->lt[l]; w->ord[l] = t->ord[l];
+        w->npos[l] = t->npos[l]; w->ncrd[l] = t->ncrd[l];
+        if (st == SP_OK) st = widen_array(t->pos[l], t->npos[l], t->posBits, stream, &w->pos[l]);
+        if (st == SP_OK) st = widen_array(t->crd[l], t->ncrd[l], t->crdBits, stream, &w->crd[l]);
+    }
+    if (st != SP_OK) { sp_free(w); return st; }
+    t->wide = w;
+    *out = w;
+    return SP_OK;
+}
+
 sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t per, cudaStream_t stream, sp_partition* out) {
     std::lock_guard<std::mutex> lock(t->mu);
     const uint64_t key = ((uint64_t)SP_PART_MTTKRP << 56) | (uint64_t)per;

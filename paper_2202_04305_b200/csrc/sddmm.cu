@@ -133,6 +133,12 @@ k_sddmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __re
 extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const double* B, int64_t ldb, int64_t K,
                               double* x_vals, void* stream_) {
     if (!S || !A || !B || K < 1 || lda < K) return SP_ERR_INVALID_ARG;
+    {   // 8- and 16-bit storage is read through its 32-bit shadow
+        sp_tensor* wide_ = nullptr;
+        const sp_status ws_ = sp_widened(S, static_cast<cudaStream_t>(stream_), &wide_);
+        if (ws_ != SP_OK) return ws_;
+        S = wide_;
+    }
     if (S->rank != 2 || S->lt[1] != SP_COMPRESSED || S->ord[0] == S->ord[1]) return SP_ERR_UNSUPPORTED;
     const bool colmajor = S->ord[0] == 1;      // S stored by columns (CSC, DCSC)
     const int64_t n = S->dims[1];

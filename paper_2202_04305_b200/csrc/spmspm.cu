@@ -45,7 +45,7 @@ __global__ void __launch_bounds__(kPThreads)
 k_spmspm(const P* __restrict__ apos, const I* __restrict__ acrd, const double* __restrict__ aval,
          const P* __restrict__ bpos, const I* __restrict__ bcrd, const double* __restrict__ bval, int64_t m,
          int64_t n, double* __restrict__ ws_all, uint32_t* __restrict__ bm_all, int64_t* __restrict__ rowlen,
-         const void* __restrict__ cpos, bool cpos64, void* __restrict__ ccrd, bool ccrd64,
+         const void* __restrict__ cpos, int cposBits, void* __restrict__ ccrd, int ccrdBits,
          double* __restrict__ cval) {
     __shared__ uint32_t sums[kPThreads / 32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -69,7 +69,7 @@ k_spmspm(const P* __restrict__ apos, const I* __restrict__ acrd, const double* _
         __syncthreads();
         // compress: bitmap words in order give the columns in order
         uint32_t carry = 0;
-        const int64_t base = NUMERIC ? (int64_t)sp_load_uint(cpos, i, cpos64) : 0;
+        const int64_t base = NUMERIC ? (int64_t)sp_load_uint(cpos, i, cposBits) : 0;
         for (int64_t w0 = 0; w0 < words; w0 += kPThreads) {
             const int64_t wi = w0 + threadIdx.x;
             uint32_t bits = wi < words ? bm[wi] : 0u;
@@ -83,7 +83,7 @@ k_spmspm(const P* __restrict__ apos, const I* __restrict__ acrd, const double* _
                         const int bpos_ = __ffs(bits) - 1;
                         bits &= bits - 1;
                         const int64_t j = (wi << 5) + bpos_;
-                        sp_store_uint(ccrd, slot, (uint64_t)j, ccrd64);
+                        sp_store_uint(ccrd, slot, (uint64_t)j, ccrdBits);
                         cval[slot] = ws[j];
                         ws[j] = 0.0;
                         ++slot;
@@ -99,11 +99,11 @@ k_spmspm(const P* __restrict__ apos, const I* __restrict__ acrd, const double* _
 
 // Single block: pos[0] = 0, pos[i+1] = rowlen[0] + .. + rowlen[i]; total to *count.
 __global__ void __launch_bounds__(kPThreads)
-k_row_offsets(const int64_t* __restrict__ rowlen, int64_t m, void* __restrict__ pos, bool pos64, int64_t* __restrict__ count) {
+k_row_offsets(const int64_t* __restrict__ rowlen, int64_t m, void* __restrict__ pos, int posBits, int64_t* __restrict__ count) {
     __shared__ unsigned long long s_w[kPThreads / 32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     unsigned long long run = 0;
-    if (threadIdx.x == 0) sp_store_uint(pos, 0, 0, pos64);
+    if (threadIdx.x == 0) sp_store_uint(pos, 0, 0, posBits);
     for (int64_t b = 0; b < m; b += kPThreads) {
         const int64_t i = b + threadIdx.x;
         unsigned long long v = i < m ? (unsigned long long)rowlen[i] : 0ull, incl = v;
@@ -117,7 +117,7 @@ k_row_offsets(const int64_t* __restrict__ rowlen, int64_t m, void* __restrict__ 
         unsigned long long pre = 0, tot = 0;
         for (int q = 0; q < kPThreads / 32; ++q) { if (q < w) pre += s_w[q]; tot += s_w[q]; }
         __syncthreads();
-        if (i < m) sp_store_uint(pos, i + 1, run + pre + incl, pos64);
+        if (i < m) sp_store_uint(pos, i + 1, run + pre + incl, posBits);
         run += tot;
     }
     if (threadIdx.x == 0) *count = (int64_t)run;
@@ -132,7 +132,14 @@ extern "C" sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBi
     if (!A || !B) return SP_ERR_INVALID_ARG;
     if (posBits == 0) posBits = 64;
     if (crdBits == 0) crdBits = 64;
-    if ((posBits != 32 && posBits != 64) || (crdBits != 32 && crdBits != 64)) return SP_ERR_INVALID_ARG;
+    if (!sp_valid_width(posBits) || !sp_valid_width(crdBits)) return SP_ERR_INVALID_ARG;
+    {   // 8- and 16-bit operands are read through their 32-bit shadows (a cache inside the handle)
+        sp_tensor *wa = nullptr, *wb = nullptr;
+        sp_status ws_ = sp_widened(const_cast<sp_tensor*>(A), static_cast<cudaStream_t>(stream_), &wa);
+        if (ws_ == SP_OK) ws_ = sp_widened(const_cast<sp_tensor*>(B), static_cast<cudaStream_t>(stream_), &wb);
+        if (ws_ != SP_OK) return ws_;
+        A = wa; B = wb;
+    }
     auto is_csr = [](const sp_tensor* t) {
         return t->rank == 2 && t->lt[0] == SP_DENSE && t->lt[1] == SP_COMPRESSED && t->ord[0] == 0 && t->ord[1] == 1;
     };
@@ -141,7 +148,7 @@ extern "C" sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBi
     if (A->dims[1] != B->dims[0]) return SP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int64_t m = A->dims[0], n = B->dims[1];
-    if (crdBits == 32 && (uint64_t)(n - 1) > 0xffffffffull) return SP_ERR_WIDTH_OVERFLOW;
+    if (n > 0 && (uint64_t)(n - 1) > sp_width_max(crdBits)) return SP_ERR_WIDTH_OVERFLOW;
 
     int64_t nblocks = m < 148 * 4 ? m : 148 * 4;
     if (nblocks < 1) nblocks = 1;
@@ -172,17 +179,17 @@ extern "C" sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBi
         k_spmspm<P, I, NUM><<<(unsigned)nblocks, kPThreads, 0, stream>>>(                                         \
             static_cast<const P*>(A->pos[1]), static_cast<const I*>(A->crd[1]), A->val,                           \
             static_cast<const P*>(B->pos[1]), static_cast<const I*>(B->crd[1]), B->val, m, n, wsrow, bm, rowlen,  \
-            C->pos[1], posBits == 64, C->crd[1], crdBits == 64, C->val);                                          \
+            C->pos[1], posBits, C->crd[1], crdBits, C->val);                                          \
     })
     if (m > 0) SP_SPMSPM_LAUNCH(false);
-    k_row_offsets<<<1, kPThreads, 0, stream>>>(rowlen, m, C->pos[1], posBits == 64, d_count);
+    k_row_offsets<<<1, kPThreads, 0, stream>>>(rowlen, m, C->pos[1], posBits, d_count);
     if (cudaGetLastError() != cudaSuccess) return fail(SP_ERR_CUDA);
     sp_count_launches(2);
     int64_t count = 0;
     if (cudaMemcpyAsync(&count, d_count, sizeof count, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
         cudaStreamSynchronize(stream) != cudaSuccess)
         return fail(SP_ERR_CUDA);
-    if (posBits == 32 && (uint64_t)count > 0xffffffffull) return fail(SP_ERR_WIDTH_OVERFLOW);
+    if ((uint64_t)count > sp_width_max(posBits)) return fail(SP_ERR_WIDTH_OVERFLOW);
     C->ncrd[1] = count;
     C->nval = count;
     C->crd[1] = sp_dev_alloc((size_t)(count ? count : 1) * (crdBits / 8), stream);

@@ -467,6 +467,12 @@ bool matrix_encoding_ok(const sp_tensor* A) {
 
 extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* stream_) {
     if (!A || !x || !y) return SP_ERR_INVALID_ARG;
+    {   // 8- and 16-bit storage is read through its 32-bit shadow
+        sp_tensor* wide_ = nullptr;
+        const sp_status ws_ = sp_widened(A, static_cast<cudaStream_t>(stream_), &wide_);
+        if (ws_ != SP_OK) return ws_;
+        A = wide_;
+    }
     if (A->rank == 2 && A->lt[1] == SP_DENSE && A->ord[0] != A->ord[1])
         return sp_spmv_dense_inner(A, x, y, static_cast<cudaStream_t>(stream_));
     if (!matrix_encoding_ok(A)) return SP_ERR_UNSUPPORTED;
@@ -505,6 +511,12 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
                              void* stream_) {
     if (!A || !B || !C || N < 1 || ldb < N || ldc < N) return SP_ERR_INVALID_ARG;
     if (N >= (1 << 20)) return SP_ERR_UNSUPPORTED;
+    {   // 8- and 16-bit storage is read through its 32-bit shadow
+        sp_tensor* wide_ = nullptr;
+        const sp_status ws_ = sp_widened(A, static_cast<cudaStream_t>(stream_), &wide_);
+        if (ws_ != SP_OK) return ws_;
+        A = wide_;
+    }
     if (A->rank == 2 && A->lt[1] == SP_DENSE && A->ord[0] != A->ord[1])
         return sp_spmm_dense_inner(A, B, N, ldb, C, ldc, static_cast<cudaStream_t>(stream_));
     if (!matrix_encoding_ok(A)) return SP_ERR_UNSUPPORTED;
@@ -630,6 +642,7 @@ __global__ void k_static_partition(const P* __restrict__ pos, int64_t nseg, int6
 extern "C" sp_status sp_spmv_static(const sp_tensor* A, const double* x, double* y, void* stream_) {
     if (!A || !x || !y) return SP_ERR_INVALID_ARG;
     if (!matrix_encoding_ok(A)) return SP_ERR_UNSUPPORTED;
+    if (A->posBits < 32 || A->crdBits < 32) return SP_ERR_UNSUPPORTED;   // a widened copy would need an allocation
     const int64_t nseg = A->npos[1] - 1;
     const int64_t nnz = A->ncrd[1];
     if (nseg + nnz > (int64_t)SP_SPMV_STATIC_MAX_ITEMS) return SP_ERR_TOO_LARGE;

@@ -62,12 +62,16 @@ extern "C" sp_status sp_vec_dot(const sp_tensor* a, const sp_tensor* b, double* 
     if (a->ncrd[0] > b->ncrd[0]) { const sp_tensor* t = a; a = b; b = t; }    // walk the shorter one
     if (a->ncrd[0] == 0) return SP_OK;
     const unsigned blocks = (unsigned)sp_ceil_div(a->ncrd[0], 256);
-    if (a->crdBits == 32)
-        k_vec_dot<uint32_t><<<blocks, 256, 0, stream>>>(static_cast<const uint32_t*>(a->crd[0]), a->val, a->ncrd[0],
-                                                       static_cast<const uint32_t*>(b->crd[0]), b->val, b->ncrd[0], result);
-    else
-        k_vec_dot<uint64_t><<<blocks, 256, 0, stream>>>(static_cast<const uint64_t*>(a->crd[0]), a->val, a->ncrd[0],
-                                                       static_cast<const uint64_t*>(b->crd[0]), b->val, b->ncrd[0], result);
+#define SP_VEC_DOT(I)                                                                                             \
+    k_vec_dot<I><<<blocks, 256, 0, stream>>>(static_cast<const I*>(a->crd[0]), a->val, a->ncrd[0],                \
+                                             static_cast<const I*>(b->crd[0]), b->val, b->ncrd[0], result)
+    switch (a->crdBits) {
+        case 8: SP_VEC_DOT(uint8_t); break;
+        case 16: SP_VEC_DOT(uint16_t); break;
+        case 32: SP_VEC_DOT(uint32_t); break;
+        default: SP_VEC_DOT(uint64_t); break;
+    }
+#undef SP_VEC_DOT
     SP_LAUNCH_CHECK();
     sp_count_launches(1);
     return SP_OK;

@@ -3,7 +3,7 @@ tensor, check that all results agree, and rank the encodings by time.
 
 The paper's loop enumerates level types x dimension orderings x pointer widths x index widths and
 calls verify(result) on each; this is the same loop over the encodings the library executes
-(bit widths 32 and 64), with the agreement check between encodings taking the place of verify."""
+(bit widths 8 to 64; a width the tensor overflows is skipped), with the agreement check between encodings taking the place of verify."""
 from __future__ import annotations
 
 import itertools
@@ -15,7 +15,7 @@ from . import binding as sp
 
 LEVELS_2D = [(sp.DENSE, sp.DENSE), (sp.DENSE, sp.COMPRESSED), (sp.COMPRESSED, sp.DENSE), (sp.COMPRESSED, sp.COMPRESSED)]
 ORDERINGS_2D = [(0, 1), (1, 0)]
-WIDTHS = [32, 64]
+WIDTHS = [8, 16, 32, 64]
 
 
 def _time(fn, reps):

@@ -25,8 +25,11 @@ def dev(a):
 
 
 def unsigned(t):
+    """Overhead array of any width (8/16-bit unsigned, 32/64-bit words viewed as signed) as int64 values."""
+    if t.numel() == 0:
+        return np.empty(0, np.int64)
     a = t.cpu().numpy()
-    return a.view(np.uint32 if a.dtype == np.int32 else np.uint64).astype(np.int64) if a.size else a.astype(np.int64)
+    return a.view({1: np.uint8, 2: np.uint16, 4: np.uint32, 8: np.uint64}[a.dtype.itemsize]).astype(np.int64)
 
 
 def assert_storage_equal(t, ref):

@@ -103,7 +103,7 @@ def test_error_codes():
         b.sp_pack(coo.dims, c, v, (0, 1), (0, 0))
     assert e.value.code == 1
     with pytest.raises(b.SpError) as e:
-        b.sp_pack(coo.dims, c, v, (0, 1), None, 16, 32)
+        b.sp_pack(coo.dims, c, v, (0, 1), None, 12, 32)
     assert e.value.code == 1
     with pytest.raises(b.SpError) as e:           # 2^33 columns do not fit 32-bit coordinates
         b.sp_pack((4, 1 << 33), c, v, (0, 1), None, 32, 32)

@@ -45,9 +45,16 @@ def test_state_space_search_over_encodings():
     coo = I.row_band_matrix(600, 20, seed=2)
     coords, vals = to_dev(coo)
     x = torch.as_tensor(I.uniform_pm1(2, 3, 600), device="cuda")
-    ranked = search.search_matrix_kernel(coo.dims, coords, vals, lambda h: sp().sp_spmv(h, x), reps=2)
+    ranked = search.search_matrix_kernel(coo.dims, coords, vals, lambda h: sp().sp_spmv(h, x), widths=[32, 64], reps=2)
     assert len(ranked) == 4 * 2 * 4                     # all level types x orderings x width pairs ran and agreed
     assert all(r["max_dev"] <= 1e-9 for r in ranked)
+    # with the narrow widths too: 600 > 2^8 rules 8-bit coordinates out wherever a level is compressed, and
+    # 12 000 entries rule 8-bit positions out; (dense, dense) stores no overhead and takes any width
+    ranked = search.search_matrix_kernel(coo.dims, coords, vals, lambda h: sp().sp_spmv(h, x), reps=1)
+    combos = {(r["levels"], r["posBits"], r["crdBits"]) for r in ranked}
+    assert ((0, 0), 8, 8) in combos and ((0, 1), 16, 16) in combos
+    assert not any(lt != (0, 0) and cb == 8 for lt, _, cb in combos)
+    assert not any(lt[1] == 1 and pb == 8 for lt, pb, _ in combos)
     B = torch.as_tensor(I.dense_operand(2, 4, 600, 8), device="cuda")
     ranked = search.search_matrix_kernel(coo.dims, coords, vals, lambda h: sp().sp_spmm(h, B), widths=[32], reps=2)
     assert len(ranked) == 8

@@ -139,3 +139,19 @@ def test_empty(oracle):
     assert s.pos[1].tolist() == [0] * 5 and s.crd[1].size == 0 and s.val.size == 0
     s = oracle.pack((4, 5), [[], []], [], (1, 1))
     assert s.pos[0].tolist() == [0, 0] and s.pos[1].tolist() == [0]
+
+
+def test_min_widths_follow_the_largest_position_and_level_size(oracle):
+    # Section 4.1: a width must hold the largest position / coordinate.  Hand-computed cases:
+    # 255 entries in a 256-long vector fit 8 bits; 256 entries need 16-bit positions; a level of
+    # size 257 needs 16-bit coordinates even if only coordinate 0 is stored.
+    v = oracle.pack((256,), [np.arange(255)], np.ones(255), (1,))
+    assert oracle.min_widths(v) == (8, 8)
+    v = oracle.pack((256,), [np.arange(256)], np.ones(256), (1,))
+    assert oracle.min_widths(v) == (16, 8)
+    v = oracle.pack((257,), [np.zeros(1, np.int64)], np.ones(1), (1,))
+    assert oracle.min_widths(v) == (8, 16)
+    m = oracle.pack((3, 1 << 33), [np.array([0, 2]), np.array([5, 1 << 32])], np.ones(2), (0, 1))
+    assert oracle.min_widths(m) == (8, 64)
+    d = oracle.pack((300, 300), [np.array([0]), np.array([0])], np.ones(1), (0, 0))
+    assert oracle.min_widths(d) == (8, 8)          # dense levels store no overhead at all
