@@ -168,8 +168,9 @@ sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t ldb,
 
 /*
  * sp_sddmm - X[i,j] = S[i,j] * sum_k A[i,k] * B[k,j] for the stored (i,j) of
- * S (Section 6.2).  S: rank 2, (dense|compressed, compressed), either
- * ordering (CSR, DCSR, CSC, DCSC).  A is dims[0] x K (lda), B is K x dims[1] (ldb).  x_vals receives
+ * S (Section 6.2).  S: rank 2, any of the eight encodings (for a dense inner
+ * level every cell of a stored row or column counts as stored, explicit zeros
+ * included).  A is dims[0] x K (lda), B is K x dims[1] (ldb).  x_vals receives
  * one value per stored entry of S, in S's storage order (X shares S's
  * positions and coordinates); its length is sp_values' len.
  */

@@ -1,6 +1,7 @@
 // sp_sddmm: X[i,j] = S[i,j] * sum_k A[i,k] * B[k,j] over the stored (i,j) of S
-// (Section 6.2), S in (dense|compressed, compressed) storage, row- or column-major.
+// (Section 6.2), S in any two-dimensional encoding, row- or column-major.
 //
+// Compressed inner level (CSR, DCSR, CSC, DCSC):
 // Loop shape: for each stored row i, for each p in pos[1][q]..pos[1][q+1]:
 // j = crd[1][p]; x[p] = S.val[p] * dot(A[i,:], B[:,j]).  B is given K x n row-major,
 // so a column is K elements a whole row apart; it is transposed once per call into
@@ -128,6 +129,79 @@ k_sddmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __re
     if (nzbase + lane < j1) xv[nzbase + lane] = v_l * res;
 }
 
+// S with a dense inner level ((dense|compressed, dense), either ordering): every cell of a stored
+// outer index is a stored value, so x[q * ninner + c] = S.val[..] * sum_k Out[o,k] * In[k,c] with
+// o the outer coordinate of stored row q.  One thread per inner coordinate c (loads of In[k, c..]
+// coalesce, Out[o,k] is a broadcast), kDQ stored outer rows per block share each load of In.
+constexpr int kDQ = 4;
+
+template <typename I>
+__global__ void __launch_bounds__(256)
+k_sddmm_dense_inner(const I* __restrict__ outer, int64_t nouter, int64_t ninner, const double* __restrict__ sval,
+                    const double* __restrict__ Out, int64_t out_row_stride, int64_t out_k_stride,
+                    const double* __restrict__ In, int64_t ldin, int64_t K, double* __restrict__ xv) {
+    const int64_t c = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    for (int64_t q0 = (int64_t)blockIdx.y * kDQ; q0 < nouter; q0 += (int64_t)gridDim.y * kDQ) {
+        const double* orow[kDQ];
+        double acc[kDQ];
+#pragma unroll
+        for (int r = 0; r < kDQ; ++r) {
+            const int64_t q = q0 + r < nouter ? q0 + r : nouter - 1;
+            orow[r] = Out + (outer ? (int64_t)outer[q] : q) * out_row_stride;
+            acc[r] = 0.0;
+        }
+        if (c < ninner) {
+            for (int64_t k = 0; k < K; ++k) {
+                const double b = In[k * ldin + c];
+#pragma unroll
+                for (int r = 0; r < kDQ; ++r) acc[r] = fma(orow[r][k * out_k_stride], b, acc[r]);
+            }
+#pragma unroll
+            for (int r = 0; r < kDQ; ++r) {
+                const int64_t p = (q0 + r) * ninner + c;
+                if (q0 + r < nouter) xv[p] = sval[p] * acc[r];
+            }
+        }
+    }
+}
+
+sp_status sddmm_dense_inner(sp_tensor* S, const double* A, int64_t lda, const double* B, int64_t ldb, int64_t K,
+                            double* x_vals, cudaStream_t stream) {
+    if (S->nval == 0) return SP_OK;
+    if (!x_vals) return SP_ERR_INVALID_ARG;
+    const bool colmajor = S->ord[0] == 1;
+    const bool dbl = S->lt[0] == SP_COMPRESSED;
+    const int64_t ninner = S->dims[S->ord[1]];
+    const int64_t nouter = dbl ? S->ncrd[0] : S->dims[S->ord[0]];
+    if (nouter == 0 || ninner == 0) return SP_OK;
+    sp_workspace ws(stream);
+    const double *Out = A, *In = B;
+    int64_t out_row = lda, out_k = 1, ldin = ldb;
+    if (colmajor) {
+        // outer = column j: Out[j,k] = B[k,j]; inner = row i: In[k,i] = A[i,k], transposed once so that
+        // neighbouring threads read neighbouring addresses
+        const int64_t m = S->dims[0];
+        double* At = ws.get<double>((size_t)K * m);
+        if (ws.failed) return SP_ERR_ALLOC;
+        dim3 tg((unsigned)sp_ceil_div(K, 32), (unsigned)sp_ceil_div(m, 32));
+        k_transpose<<<tg, 256, 0, stream>>>(A, lda, m, K, At, m);
+        SP_LAUNCH_CHECK();
+        sp_count_launches(1);
+        Out = B; out_row = 1; out_k = ldb;
+        In = At; ldin = m;
+    }
+    dim3 grid((unsigned)sp_ceil_div(ninner, 256), (unsigned)std::min<int64_t>(sp_ceil_div(nouter, kDQ), 32768));
+    if (S->crdBits == 32)
+        k_sddmm_dense_inner<uint32_t><<<grid, 256, 0, stream>>>(dbl ? static_cast<const uint32_t*>(S->crd[0]) : nullptr, nouter,
+                                                               ninner, S->val, Out, out_row, out_k, In, ldin, K, x_vals);
+    else
+        k_sddmm_dense_inner<uint64_t><<<grid, 256, 0, stream>>>(dbl ? static_cast<const uint64_t*>(S->crd[0]) : nullptr, nouter,
+                                                               ninner, S->val, Out, out_row, out_k, In, ldin, K, x_vals);
+    SP_LAUNCH_CHECK();
+    sp_count_launches(1);
+    return SP_OK;
+}
+
 }  // namespace
 
 extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const double* B, int64_t ldb, int64_t K,
@@ -139,7 +213,9 @@ extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const 
         if (ws_ != SP_OK) return ws_;
         S = wide_;
     }
-    if (S->rank != 2 || S->lt[1] != SP_COMPRESSED || S->ord[0] == S->ord[1]) return SP_ERR_UNSUPPORTED;
+    if (S->rank != 2 || S->ord[0] == S->ord[1]) return SP_ERR_UNSUPPORTED;
+    if (ldb < S->dims[1]) return SP_ERR_INVALID_ARG;
+    if (S->lt[1] == SP_DENSE) return sddmm_dense_inner(S, A, lda, B, ldb, K, x_vals, static_cast<cudaStream_t>(stream_));
     const bool colmajor = S->ord[0] == 1;      // S stored by columns (CSC, DCSC)
     const int64_t n = S->dims[1];
     if (ldb < n) return SP_ERR_INVALID_ARG;

@@ -140,10 +140,6 @@ def test_unsupported_encodings():
     b = sp()
     coo = I.uniform_matrix(20, 20, 50, seed=1)
     coords, vals = to_dev(coo)
-    A = b.sp_pack(coo.dims, coords, vals, (1, 0))
-    with pytest.raises(b.SpError) as e:
-        b.sp_sddmm(A, dev(np.ones((20, 4))), dev(np.ones((4, 20))))
-    assert e.value.code == 2
     T = b.sp_pack((20, 20, 1), coords + [coords[0] * 0], vals, (1, 1, 1))
     with pytest.raises(b.SpError) as e:
         b.sp_spmv(T, dev(np.ones(20)))
@@ -274,6 +270,25 @@ def test_sddmm_column_major_sample(oracle, enc, K):
         ref = np.empty_like(xe); bd = np.empty_like(be)
         ref[ep] = xe; bd[ep] = be
         assert_close(xg, ref, bd, f"sddmm {enc} {name} K={K}")
+
+
+@pytest.mark.parametrize("lt", [(1, 0), (0, 0)])
+@pytest.mark.parametrize("od", [(0, 1), (1, 0)])
+@pytest.mark.parametrize("K", [1, 7, 64, 130])
+def test_sddmm_dense_inner_level(oracle, lt, od, K):
+    # S with a dense inner level: every cell of a stored row (column) is a stored value, explicit zeros included
+    for name, coo in [("uniform", I.uniform_matrix(300, 257, 4000, seed=1)), ("band", I.row_band_matrix(270, 9, seed=4)),
+                      ("one_row", MATS[7][1]), ("empty", I.uniform_matrix(9, 9, 0, seed=1))]:
+        coords, vals = to_dev(coo)
+        S = sp().sp_pack(coo.dims, coords, vals, lt, od)
+        A = I.dense_operand(13, 8, coo.dims[0], K)
+        B = I.dense_operand(13, 9, K, coo.dims[1])
+        xg = sp().sp_sddmm(S, dev(A), dev(B)).cpu().numpy()
+        (si, sj), sv = oracle.unpack(oracle.pack(coo.dims, coo.coords, coo.vals, lt, od))   # stored cells, storage order
+        assert xg.size == sv.size
+        if sv.size:
+            ref, bd = oracle.sddmm(si, sj, sv, A, B)
+            assert_close(xg, ref, bd, f"sddmm dense inner {lt}{od} {name} K={K}")
 
 
 @pytest.mark.parametrize("mode", [0, 1, 2])
