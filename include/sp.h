@@ -29,6 +29,12 @@
  *     different algorithm on the host.
  *   - A handle is immutable after sp_pack.  Kernels cache work-partition tables
  *     inside it on first use; use a handle from one stream at a time.
+ *   - CUDA graphs: once a kernel call has run on a handle (so its cached tables
+ *     exist), later sp_spmv / sp_spmm / sp_sddmm / sp_mttkrp calls on it only
+ *     enqueue stream-ordered work and may be stream-captured, provided the
+ *     installed allocator is itself legal during capture (a stream-ordered or
+ *     caching pool; the default cudaMalloc is not).  sp_pack, sp_convert, sp_unpack
+ *     and sp_spmspm read sizes back to the host and cannot be captured.
  */
 #ifndef SP_H
 #define SP_H
