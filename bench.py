@@ -93,7 +93,42 @@ def work_model(wl):
     k["sddmm_csr"] = dict(flops=c4.nnz * (2 * K4 + 1), bytes=20 * c4.nnz + W * (c4.dims[0] + 1) + 8 * K4 * sum(c4.dims))
     k["pack_csf"] = dict(flops=0, bytes=c5.nnz * 20 + c5.nnz * 12 + 2 * W * F5, units=c5.nnz)
     k["mttkrp_csf"] = dict(flops=2 * R5 * (c5.nnz + F5), bytes=12 * c5.nnz + 2 * W * F5 + 8 * R5 * sum(c5.dims))
+    # Dense rows the method fetches per stored entry (one row of the dense operand each; no reuse assumed):
+    # rows fetched, doubles per row, rows of the table they are drawn from.
+    k["spmm_dcsr"]["gather"] = dict(rows=c3.nnz, row_elems=N3, table_rows=n3)
+    k["spmm_csr"]["gather"] = dict(rows=c2.nnz, row_elems=N2, table_rows=c2.dims[1])
+    k["sddmm_csr"]["gather"] = dict(rows=c4.nnz, row_elems=K4, table_rows=c4.dims[1])
+    k["mttkrp_csf"]["gather"] = dict(rows=c5.nnz + F5, row_elems=R5, table_rows=c5.dims[2])
     return k
+
+
+def secondary_bounds(sp, torch, model):
+    """Measured rates behind the gather kernels' second bound: random whole-row fetches from a table of the
+    operand's size (L2-resident or not) and the register-only f64 multiply-add rate."""
+    def best_ms(fn, reps=5):
+        n = fn(); torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record(); torch.cuda.synchronize()
+            best = min(best, a.elapsed_time(b))
+        return best, n
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    out = {"gather_gbs": {}}
+    for name, m in model.items():
+        g = m.get("gather")
+        if not g:
+            continue
+        key = f"{g['row_elems'] * 8}B_rows_of_{g['table_rows'] * g['row_elems'] * 8 / 1e6:.0f}MB_table"
+        if key not in out["gather_gbs"]:
+            table = torch.rand(g["table_rows"], g["row_elems"], dtype=torch.float64, device="cuda")
+            ms, n = best_ms(lambda: sp.sp_probe_gather(table, sms * 8, 1024))
+            out["gather_gbs"][key] = round(n * g["row_elems"] * 8 / (ms * 1e-3) / 1e9, 1)
+            del table
+        g["gbs"] = out["gather_gbs"][key]
+    ms, n = best_ms(lambda: sp.sp_probe_dfma(sms * 8, 20000))
+    out["dfma_tflops"] = round(2 * n / (ms * 1e-3) / 1e12, 2)
+    return out
 
 
 # --------------------------------------------------------------------------- GPU arm
@@ -403,6 +438,7 @@ def main():
     model["next_spmspm_csr"] = dict(flops=2 * products, bytes=12 * (qa.nnz + qb.nnz + qc.nval) + 4 * 3 * (qa.dims[0] + 1),
                                     units=products)
     qc.free()
+    bounds = secondary_bounds(sp, torch, model)
     for name, fn in calls.items():
         ts = suite.time_call(fn, args.kernel_reps)
         med = statistics.median(ts)
@@ -413,6 +449,15 @@ def main():
                          "frac_of_8TBs": round(gbs / 8000.0, 4)}
         if "units" in m:
             kernels[name]["Mnnz_per_s"] = round(m["units"] / (med * 1e-3) / 1e6, 1)
+        if "gather" in m:
+            # second bound: the rows the method fetches (one per stored entry) at the probed random-row rate
+            g = m["gather"]
+            gms = g["rows"] * g["row_elems"] * 8 / (g["gbs"] * 1e9) * 1e3
+            fms = m["flops"] / (bounds["dfma_tflops"] * 1e12) * 1e3
+            kernels[name].update({"gather_bytes": g["rows"] * g["row_elems"] * 8, "gather_probe_gbs": g["gbs"],
+                                  "gather_bound_ms": round(gms, 4), "dfma_bound_ms": round(fms, 4),
+                                  "hbm_bound_ms": round(m["bytes"] / (peak * 1e9) * 1e3, 4),
+                                  "frac_of_gather_bound": round(gms / med, 4)})
 
     # ---- dominant kernel: the sort's scatter pass inside sp_pack, timed by the library's own events
     sp.sp_set_profiling(True)
@@ -463,7 +508,7 @@ def main():
                 "dtype": "f64", "data": "synthetic", "config": cfg, "clocks": clocks,
                 "effective_gbs": round(world * total_bytes / (ms_step * 1e-3) / 1e9, 1),
                 "gpu_launches": int(launches), "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu,
-                "kernels": kernels, "pack_profile": prof, "peak_hbm_gbs": peak}
+                "kernels": kernels, "secondary_bounds": bounds, "pack_profile": prof, "peak_hbm_gbs": peak}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

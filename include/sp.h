@@ -286,6 +286,29 @@ int64_t sp_launch_count(void);
 sp_status sp_set_profiling(int enabled);
 sp_status sp_get_pack_profile(double* ms /* host */, int* npasses /* host, may be NULL */);
 
+/*
+ * Probes of the two secondary bounds of the gather kernels (no counterpart in the
+ * paper): SpMM, SDDMM and MTTKRP fetch one dense row per stored entry, so besides
+ * HBM they are limited by the rate at which SMs can pull randomly chosen rows of a
+ * cache-resident table, and by the f64 multiply-add rate.  Both calls enqueue one
+ * kernel on stream and return at once; the caller times them with events.
+ *
+ * sp_probe_gather: blocks x 256 threads; lane groups fetch rows_per_group (rounded
+ * up to a multiple of 8) rows each of a row-major table[rows x row_elems] (device,
+ * 16-byte aligned, caller-owned) at pseudo-random row numbers derived from seed,
+ * eight rows in flight per group, 16 bytes per lane per load.  row_elems is 16, 32,
+ * 64 or 128 doubles (else SP_ERR_UNSUPPORTED).  sink (device, blocks*256 doubles)
+ * receives per-thread sums so the loads cannot be dropped; *fetched (host, may be
+ * NULL) receives the number of rows fetched, i.e. bytes moved = *fetched * row_elems * 8.
+ *
+ * sp_probe_dfma: blocks x 256 threads each run eight independent chains of iters
+ * dependent f64 fused multiply-adds held in registers; *fmas (host, may be NULL)
+ * receives the total count (flops = 2 * *fmas).  sink as above.
+ */
+sp_status sp_probe_gather(const double* table, int64_t rows, int64_t row_elems, int64_t blocks,
+                          int64_t rows_per_group, uint64_t seed, double* sink, int64_t* fetched, void* stream);
+sp_status sp_probe_dfma(int64_t blocks, int64_t iters, double* sink, int64_t* fmas, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libsp.so")
-SOURCES = ["api.cu", "pack.cu", "partition.cu", "spmv_spmm.cu", "sddmm.cu", "mttkrp.cu", "dense_inner.cu", "spmspm.cu", "vector_ops.cu"]
+SOURCES = ["api.cu", "pack.cu", "partition.cu", "spmv_spmm.cu", "sddmm.cu", "mttkrp.cu", "dense_inner.cu", "spmspm.cu", "vector_ops.cu", "probes.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -186,6 +186,7 @@ TENSOR_ENCODINGS = {"CSF": ((1, 1, 1), (0, 1, 2)), "DSS": ((0, 1, 1), (0, 1, 2))
 
 def _tensors():
     yield "zipf", I.config5(seed=3, dim=200, nnz=40000)
+    yield "zipf_wide", I.config5(seed=11, dim=3000, nnz=120000)     # more leaf coordinates than hot-row slots
     yield "uniform", I.uniform_tensor((50, 40, 30), 3000, seed=4)
     yield "tiny", I.uniform_tensor((3, 3, 4), 5, seed=5)
     yield "empty", I.uniform_tensor((6, 5, 4), 0, seed=6)
