@@ -135,9 +135,8 @@ __device__ __forceinline__ double sp_shfl(double v, int src) {
 
 // Partition tables (partition.cu).  kind distinguishes the position array used.
 enum { SP_PART_MERGE_LAST = 1, SP_PART_MTTKRP = 2, SP_PART_SEGIDS = 3 };
-// For storage whose innermost level is compressed: the coordinate, at the level above, of every
-// stored entry (the expanded "outer" index: a matrix entry's row or column, a rank-3 entry's
-// level-1 coordinate), uint32, cached in the handle.  Needs dims < 2^32.
+// For rank-2 (x, compressed) storage: the logical level-0 coordinate of every stored entry
+// (the expanded "outer" index), uint32, cached in the handle.  Needs dims < 2^32.
 sp_status sp_get_segment_ids(sp_tensor* t, cudaStream_t stream, const uint32_t** out);
 sp_status sp_get_merge_partition(sp_tensor* t, int64_t items_per_chunk, int64_t carry_elems_per_chunk,
                                  cudaStream_t stream, sp_partition* out);

@@ -159,27 +159,28 @@ k_mttkrp(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* __rest
 
 
 // ---------------------------------------------------------------------------------------------
-// Fast path (R even, factor rows 16-byte aligned, dim * R < 2^31, dims < 2^32).
+// Fast path (R a multiple of S, factor rows 16-byte aligned, dim * R < 2^31).
 //
-// The loop nest is flattened completely: with the level-1 coordinate j of every entry at hand
-// (expanded once per handle, like the column of every entry of a column-major matrix) an entry
-// contributes val * F2[k,:] * F1[j,:] to the row of its slice, and the only structure left in the
-// hot loop is the slice boundary.  A warp walks its entry range 32 entries at a time.  Each lane
-// stages one entry of the batch - the element offsets of its two factor rows and its value - in
-// shared memory.  The warp then splits into S groups of 32/S lanes; a lane owns S adjacent output
-// columns and group g takes entries g, g+S, g+2S ... of the batch, so a group fetches a 32-column
-// factor row with S/2 16-byte loads per lane.  Consecutive entries mostly share j, so the F1 row
-// comes from L1.  There is no branch and no fibre state in the entry loop; all loads of kUnroll
-// entries per group are issued before the first multiply-add.  Batches never straddle a slice end;
-// at a slice end the groups' sums are folded with shuffles and the row is stored.
+// A warp walks its entry range 32 entries at a time.  Each lane first prepares one entry of the
+// batch - the element offset of its leaf factor row, the element offset of the level-1 factor row
+// of the fibre it lies in, and whether a fibre sum must be closed after it - and parks that in
+// shared memory.  The warp then splits into S groups of 32/S lanes; group g consumes the 32/S
+// consecutive entries g*32/S .. of the batch, and a lane owns S adjacent output columns, so a
+// group fetches a whole 32-column factor row with one (S = 2) or two (S = 4) 16-byte loads per
+// lane.  Closing a fibre is accs += F1[j,:] * accf, written branch-free (a row of zeros when no
+// close is due).  Every group closes its open partial sum at the end of its entries - sums are
+// linear, so a fibre may be closed in pieces - which keeps the inner loop free of any cross-batch
+// fibre state.  Batches never straddle a slice end.
 struct __align__(16) Staged {
-    uint32_t koff;   // leaf (level-2) factor row offset, elements
-    uint32_t joff;   // level-1 factor row offset, elements
+    uint32_t koff;   // leaf factor row offset (elements)
+    uint32_t bw;     // (level-1 factor row offset << 1) | close-after-this-entry
     double v;
 };
 
 constexpr int kFastPer = 1024;   // entries per warp
 
+// A lane's S columns are S/2 pairs; pair n sits at column offset coff[n] of the 32-column tile,
+// laid out so that the lanes of a group read one contiguous run per 16-byte load.
 template <int S>
 __device__ __forceinline__ void ld_cols(const double* p, const int* coff, double* a) {
 #pragma unroll
@@ -192,12 +193,13 @@ __device__ __forceinline__ void ld_cols(const double* p, const int* coff, double
 
 template <typename P, typename I, int S>
 __global__ void __launch_bounds__(kTThreads)
-k_mttkrp_flat(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* __restrict__ pos2,
-              const uint32_t* __restrict__ jexp, const I* __restrict__ crd2, const double* __restrict__ val,
+k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* __restrict__ pos2,
+              const I* __restrict__ crd1, const I* __restrict__ crd2, const double* __restrict__ val,
               const double* __restrict__ F1, const double* __restrict__ F2, int64_t R, double* __restrict__ M,
-              const int64_t* __restrict__ pnz, const int64_t* __restrict__ pslice, int64_t nchunks, int64_t nslice) {
-    constexpr int GL = 32 / S;      // lanes per group; a group takes every S-th entry of a batch
-    constexpr int kUnroll = 2;      // entries per group whose loads are in flight together
+              const int64_t* __restrict__ pfiber, const int64_t* __restrict__ pnz,
+              const int64_t* __restrict__ pslice, int64_t nchunks, int64_t nslice, int64_t nfiber) {
+    constexpr int GL = 32 / S;      // lanes per group = entries per group and batch
+    constexpr int kStepGroup = S == 2 ? 4 : 2;
     __shared__ Staged s_st[kTThreads / 32][32];
     __shared__ double s_car[2 * kTThreads / 32][32];
     __shared__ long long s_id[2 * kTThreads / 32];
@@ -220,93 +222,143 @@ k_mttkrp_flat(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
         }
         const double* F1g = F1 + rb;
         const double* F2g = F2 + rb;
-        int64_t s = work ? pslice[w] : 0, p = p0;
-        int64_t slice_end = work ? (int64_t)pos2[(int64_t)pos1[s + 1]] : kInf;   // entry index at which slice s ends
+        int64_t f = work ? pfiber[w] : 0, s = work ? pslice[w] : 0, p = p0, fb = f;
+        int64_t send = work ? (int64_t)pos1[s + 1] : 0;
+        int64_t slice_end = work ? (int64_t)pos2[send] : kInf;   // entry index at which slice s ends
         long long head_id = -1, tail_id = -1;
-        double acc[S];
+        double head_v[S], tail_v[S], accs[S];
 #pragma unroll
-        for (int q = 0; q < S; ++q) acc[q] = 0.0;
+        for (int q = 0; q < S; ++q) { head_v[q] = 0.0; tail_v[q] = 0.0; accs[q] = 0.0; }
         bool first = true;
         int64_t last_flush = p0;
+        // three windows of 32 fibres: ends and level-1 coordinates (the third is a prefetch)
+        int64_t feA = kInf, feB = kInf, feC = kInf;
+        I jA = 0, jB = 0, jC = 0;
+        if (work) {
+            if (fb + lane < nfiber) { feA = (int64_t)pos2[fb + lane + 1]; jA = crd1[fb + lane]; }
+            if (fb + 32 + lane < nfiber) { feB = (int64_t)pos2[fb + 32 + lane + 1]; jB = crd1[fb + 32 + lane]; }
+            if (fb + 64 + lane < nfiber) { feC = (int64_t)pos2[fb + 64 + lane + 1]; jC = crd1[fb + 64 + lane]; }
+        }
         I k_n = (p + lane < p1) ? crd2[p + lane] : (I)0;
-        uint32_t j_n = (p + lane < p1) ? jexp[p + lane] : 0u;
         double v_n = (p + lane < p1) ? val[p + lane] : 0.0;
 
-        // adds the S groups' sums into every lane, then parks the row in carry slot `slot`
-        auto fold_to_slot = [&](int slot) {
+        auto fold_groups = [&]() {       // add the S groups' slice sums into group 0's lanes
 #pragma unroll
             for (int o = GL; o < 32; o <<= 1)
 #pragma unroll
-                for (int q = 0; q < S; ++q) acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], o);
-            if (slot >= 0 && g == 0) {
-#pragma unroll
-                for (int q = 0; q < S; ++q) s_car[slot][(q / 2) * 2 * GL + 2 * hl + (q & 1)] = acc[q];
-            }
+                for (int q = 0; q < S; ++q) accs[q] += __shfl_xor_sync(0xffffffffu, accs[q], o);
         };
 
         while (p < p1) {
             int64_t lim = p1 - p;
             if (slice_end - p < lim) lim = slice_end - p;
             const int cnt = lim < 32 ? (int)lim : 32;
-            const bool valid = lane < cnt;
-            Staged st;
-            st.koff = valid ? (uint32_t)k_n * Ru : 0u;
-            st.joff = valid ? j_n * Ru : 0u;
-            st.v = valid ? v_n : 0.0;
+            const I k_l = k_n;
+            const double v_l = v_n;
             {
                 const int64_t pn = p + cnt;
                 k_n = (pn + lane < p1) ? crd2[pn + lane] : (I)0;
-                j_n = (pn + lane < p1) ? jexp[pn + lane] : 0u;
                 v_n = (pn + lane < p1) ? val[pn + lane] : 0.0;
             }
+            const int64_t relA = feA - p - 1, relB = feB - p - 1;
+            const unsigned endmask = __reduce_or_sync(
+                0xffffffffu, ((relA >= 0 && relA < cnt) ? (1u << (int)relA) : 0u) |
+                                 ((relB >= 0 && relB < cnt) ? (1u << (int)relB) : 0u));
+            const int fi = (int)(f - fb) + __popc(endmask & ((1u << lane) - 1u));
+            const I ja = __shfl_sync(0xffffffffu, jA, fi & 31);
+            const I jb = __shfl_sync(0xffffffffu, jB, fi & 31);
+            const uint32_t j = (uint32_t)(fi < 32 ? ja : jb);
+            const bool valid = lane < cnt;
+            const bool close = valid && (((endmask >> lane) & 1u) || lane == cnt - 1 || hl == GL - 1);
+            Staged st;
+            st.koff = valid ? (uint32_t)k_l * Ru : 0u;
+            st.bw = valid ? (((j * Ru) << 1) | (close ? 1u : 0u)) : 0u;
+            st.v = valid ? v_l : 0.0;
             s_st[wi][lane] = st;
             __syncwarp();
-            const Staged* mine = &s_st[wi][g];
+
+            double accf[S];
 #pragma unroll
-            for (int t0 = 0; t0 < GL; t0 += kUnroll) {
-                if (t0 * S >= cnt) break;                 // the rest of the batch is empty (warp-uniform)
-                Staged e[kUnroll];
-                double c[kUnroll][S], b[kUnroll][S];
+            for (int q = 0; q < S; ++q) accf[q] = 0.0;
+            const Staged* mine = &s_st[wi][g * GL];
 #pragma unroll
-                for (int u = 0; u < kUnroll; ++u) {
-                    e[u] = mine[(t0 + u) * S];
+            for (int t0 = 0; t0 < GL; t0 += kStepGroup) {
+                // Note: no double is set to a constant zero in this loop.  Zeroing a 64-bit register
+                // pair is issued on a narrow pipe that saturates long before the loads do; a closed
+                // sum is cleared by masking its bits with integer ops instead, and the level-1 row is
+                // read only under the same predicate that consumes it.
+                Staged e[kStepGroup];
+                double c[kStepGroup][S], b[kStepGroup][S];
+#pragma unroll
+                for (int u = 0; u < kStepGroup; ++u) {
+                    e[u] = mine[t0 + u];
                     ld_cols<S>(F2g + e[u].koff, coff, c[u]);
-                    ld_cols<S>(F1g + e[u].joff, coff, b[u]);
+                    if (e[u].bw & 1u) ld_cols<S>(F1g + (e[u].bw >> 1), coff, b[u]);
                 }
 #pragma unroll
-                for (int u = 0; u < kUnroll; ++u)
+                for (int u = 0; u < kStepGroup; ++u) {
+                    const bool cl = e[u].bw & 1u;
+                    const long long keep = (long long)(int)((e[u].bw & 1u) - 1u);   // all ones, or 0 after a close
 #pragma unroll
-                    for (int q = 0; q < S; ++q) acc[q] = fma(e[u].v * c[u][q], b[u][q], acc[q]);
+                    for (int q = 0; q < S; ++q) {
+                        accf[q] = fma(e[u].v, c[u][q], accf[q]);
+                        if (cl) accs[q] = fma(b[u][q], accf[q], accs[q]);
+                        accf[q] = __longlong_as_double(__double_as_longlong(accf[q]) & keep);
+                    }
+                }
             }
             __syncwarp();
+            f += __popc(endmask);
             p += cnt;
             if (p == slice_end) {                    // slice s is complete: all groups' sums -> row i
+                fold_groups();
                 const int64_t i = crd0 ? (int64_t)crd0[s] : s;
-                fold_to_slot(first ? 2 * wi : -1);
                 if (first) {
                     head_id = i;
+#pragma unroll
+                    for (int q = 0; q < S; ++q) head_v[q] = accs[q];
                 } else if (g == 0) {
 #pragma unroll
                     for (int q = 0; q < S; q += 2)
                         if (on[q / 2])
-                            *reinterpret_cast<double2*>(M + i * R + rb + coff[q / 2]) = make_double2(acc[q], acc[q + 1]);
+                            *reinterpret_cast<double2*>(M + i * R + rb + coff[q / 2]) = make_double2(accs[q], accs[q + 1]);
                 }
                 first = false;
                 last_flush = p;
 #pragma unroll
-                for (int q = 0; q < S; ++q) acc[q] = 0.0;
-                if (p < p1) {                        // the slice that holds entry p: the next one with fibres
-                    int64_t fend = (int64_t)pos1[s + 1];
-                    ++s;
-                    while (s < nslice && (int64_t)pos1[s + 1] == fend) ++s;
-                    slice_end = s < nslice ? (int64_t)pos2[(int64_t)pos1[s + 1]] : kInf;
-                }
+                for (int q = 0; q < S; ++q) accs[q] = 0.0;
+                ++s;
+                while (s < nslice && (int64_t)pos1[s + 1] == f) ++s;   // slices with no fibres
+                if (s < nslice) { send = (int64_t)pos1[s + 1]; slice_end = (int64_t)pos2[send]; }
+                else slice_end = kInf;
+            }
+            if (f - fb >= 32) {
+                fb += 32;
+                feA = feB; jA = jB; feB = feC; jB = jC;
+                feC = kInf; jC = 0;
+                if (fb + 64 + lane < nfiber) { feC = (int64_t)pos2[fb + 64 + lane + 1]; jC = crd1[fb + 64 + lane]; }
             }
         }
         if (p1 > last_flush) {                       // the range ends inside slice s
+            fold_groups();
             const int64_t i = crd0 ? (int64_t)crd0[s] : s;
-            fold_to_slot(first ? 2 * wi : 2 * wi + 1);
-            if (first) head_id = i; else tail_id = i;
+            if (first) {
+                head_id = i;
+#pragma unroll
+                for (int q = 0; q < S; ++q) head_v[q] = accs[q];
+            } else {
+                tail_id = i;
+#pragma unroll
+                for (int q = 0; q < S; ++q) tail_v[q] = accs[q];
+            }
+        }
+        if (g == 0) {
+#pragma unroll
+            for (int q = 0; q < S; ++q) {
+                const int cc = (q / 2) * 2 * GL + 2 * hl + (q & 1);
+                s_car[2 * wi][cc] = head_v[q];
+                s_car[2 * wi + 1][cc] = tail_v[q];
+            }
         }
         if (lane == 0) { s_id[2 * wi] = head_id; s_id[2 * wi + 1] = tail_id; }
         __syncthreads();
@@ -369,22 +421,18 @@ static sp_status mttkrp_levels(sp_tensor* T, const double* F1, const double* F2,
     if (nnz == 0) return SP_OK;
     const int64_t d1 = T->dims[T->ord[1]], d2 = T->dims[T->ord[2]];
     const int64_t maxdim = d1 > d2 ? d1 : d2;
-    const bool fast = (R % 2 == 0) && maxdim * R < ((int64_t)1 << 31) && d1 < ((int64_t)1 << 32) &&
-                      reinterpret_cast<uintptr_t>(B) % 16 == 0 && reinterpret_cast<uintptr_t>(C) % 16 == 0 &&
-                      reinterpret_cast<uintptr_t>(M) % 16 == 0;
+    const bool fast = (R % 2 == 0) && maxdim * R < ((int64_t)1 << 31) && reinterpret_cast<uintptr_t>(B) % 16 == 0 &&
+                      reinterpret_cast<uintptr_t>(C) % 16 == 0 && reinterpret_cast<uintptr_t>(M) % 16 == 0;
     sp_partition part;
     sp_status st = sp_get_mttkrp_partition(T, fast ? kFastPer : kTPer, stream, &part);
     if (st != SP_OK) return st;
     const unsigned blocks = (unsigned)sp_ceil_div(part.nchunks * 32, kTThreads);
     if (fast) {
-        const uint32_t* jexp = nullptr;      // level-1 coordinate of every entry
-        st = sp_get_segment_ids(T, stream, &jexp);
-        if (st != SP_OK) return st;
 #define SP_MTTKRP_FAST(S)                                                                                              \
-    k_mttkrp_flat<P, I, S><<<blocks, kTThreads, 0, stream>>>(                                                          \
+    k_mttkrp_fast<P, I, S><<<blocks, kTThreads, 0, stream>>>(                                                          \
         static_cast<const P*>(T->pos[1]), T->lt[0] == SP_COMPRESSED ? static_cast<const I*>(T->crd[0]) : nullptr,      \
-        static_cast<const P*>(T->pos[2]), jexp, static_cast<const I*>(T->crd[2]), T->val,                              \
-        F1, F2, R, M, part.nz, part.aux, part.nchunks, T->npos[1] - 1)
+        static_cast<const P*>(T->pos[2]), static_cast<const I*>(T->crd[1]), static_cast<const I*>(T->crd[2]), T->val,  \
+        F1, F2, R, M, part.row, part.nz, part.aux, part.nchunks, T->npos[1] - 1, T->ncrd[1])
         SP_DISPATCH_WIDTHS(T, {
             if (R % 4 == 0) SP_MTTKRP_FAST(4); else SP_MTTKRP_FAST(2);
         });

@@ -372,8 +372,7 @@ struct EmitArgs {
     void* pos[SP_MAX_RANK];
     void* crd[SP_MAX_RANK];
     double* val;
-    uint32_t* seg_out;   // optional: coordinate at level seg_level of every stored entry
-    int seg_level;       // (column-major matrices: level 0; rank-3 all-compressed inner levels: level 1)
+    uint32_t* seg_out;   // optional: level-0 coordinate of every stored entry (column-major matrices)
     int posBits, crdBits;
     unsigned flags;
     int* err;
@@ -453,8 +452,7 @@ __global__ void __launch_bounds__(kCtThreads) k_emit(EmitArgs a) {
             if (dup)
                 for (int64_t g = e + 1; g < a.n && a.keys[g] == k[i]; ++g) s += a.vals_in[a.idx[g]];
             a.val[ppos] = s;
-            if (a.seg_out)
-                a.seg_out[ppos] = (uint32_t)((k[i] >> p.shift[a.seg_level]) & ((1ull << p.bits[a.seg_level]) - 1ull));
+            if (a.seg_out) a.seg_out[ppos] = (uint32_t)(k[i] >> p.shift[0]);
         } else if (a.flags & SP_DUP_ERROR) {
             atomicOr(a.err, kErrDup);
         }
@@ -776,12 +774,8 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
         a.val = t->val; a.posBits = posBits; a.crdBits = crdBits; a.flags = flags; a.err = d_err;
         // Column-major matrices run SpMM as a flat loop over entries and need each entry's column:
         // it is in the sorted key anyway, so it is written here instead of being searched for later.
-        // MTTKRP reads the level-1 coordinate of every entry of a rank-3 tensor the same way.
         a.seg_out = nullptr;
-        a.seg_level = rank - 2;
-        const bool seg_matrix = rank == 2 && plan.src[0] == 1 && plan.lt[1] == SP_COMPRESSED;
-        const bool seg_tensor = rank == 3 && plan.lt[1] == SP_COMPRESSED && plan.lt[2] == SP_COMPRESSED;
-        if ((seg_matrix || seg_tensor) && plan.sz[rank - 2] < ((int64_t)1 << 32)) {
+        if (rank == 2 && plan.src[0] == 1 && plan.lt[1] == SP_COMPRESSED && plan.sz[0] < ((int64_t)1 << 32)) {
             sp_partition sg;
             sg.aux = static_cast<int64_t*>(sp_dev_alloc((size_t)(t->nval ? t->nval : 1) * sizeof(uint32_t), stream));
             if (!sg.aux) return fail(SP_ERR_ALLOC);

@@ -46,9 +46,8 @@ __global__ void k_mttkrp_partition(const P* __restrict__ pos1, int64_t nslice, c
     nz[w] = p; fiber[w] = f; slice[w] = lo;
 }
 
-// One thread per stored entry of the innermost level: the node of the level above that holds it,
-// by binary search in the innermost pos[], mapped through that level's crd[] when it is compressed
-// (a matrix: the row or column of every entry; a rank-3 tensor: the level-1 coordinate of every entry).
+// One thread per stored entry: the segment (level-0 node) that holds it, by binary search in pos[1],
+// mapped through crd[0] when level 0 is compressed.
 template <typename P, typename I>
 __global__ void k_segment_ids(const P* __restrict__ pos, int64_t nseg, int64_t nnz, const I* __restrict__ outer,
                               uint32_t* __restrict__ seg) {
@@ -69,8 +68,7 @@ sp_status sp_get_segment_ids(sp_tensor* t, cudaStream_t stream, const uint32_t**
     const uint64_t key = (uint64_t)SP_PART_SEGIDS << 56;
     auto it = t->parts.find(key);
     if (it != t->parts.end()) { *out = reinterpret_cast<const uint32_t*>(it->second.aux); return SP_OK; }
-    const int last = t->rank - 1;           // the innermost level and the level above it
-    const int64_t nseg = t->npos[last] - 1, nnz = t->ncrd[last];
+    const int64_t nseg = t->npos[1] - 1, nnz = t->ncrd[1];
     sp_partition p;
     p.aux = static_cast<int64_t*>(sp_dev_alloc((size_t)(nnz ? nnz : 1) * sizeof(uint32_t), stream));
     if (!p.aux) return SP_ERR_ALLOC;
@@ -78,9 +76,9 @@ sp_status sp_get_segment_ids(sp_tensor* t, cudaStream_t stream, const uint32_t**
     if (nnz > 0) {
         const unsigned blocks = (unsigned)sp_ceil_div(nnz, 256);
         SP_DISPATCH_WIDTHS(t, {
-            k_segment_ids<P, I><<<blocks, 256, 0, stream>>>(
-                static_cast<const P*>(t->pos[last]), nseg, nnz,
-                t->lt[last - 1] == SP_COMPRESSED ? static_cast<const I*>(t->crd[last - 1]) : nullptr, seg);
+            k_segment_ids<P, I><<<blocks, 256, 0, stream>>>(static_cast<const P*>(t->pos[1]), nseg, nnz,
+                                                           t->lt[0] == SP_COMPRESSED ? static_cast<const I*>(t->crd[0]) : nullptr,
+                                                           seg);
         });
         SP_LAUNCH_CHECK();
         sp_count_launches(1);
