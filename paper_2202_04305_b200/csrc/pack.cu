@@ -152,7 +152,10 @@ k_sort_upsweep(const uint64_t* __restrict__ keys, int64_t n, int shift, uint32_t
 }
 
 // Lanes of the warp whose 9-bit value (digit, or kRadix for padding) equals this lane's, by one
-// ballot per bit.  (A hardware match instruction does the same but costs far more per call.)
+// ballot per bit.  The hardware match instruction does the same but costs more per call the more
+// distinct values the warp holds: with uniform 8-bit digits the scatter pass ran 0.31 ms per five
+// passes over 5 M entries with it and 0.24 ms with the ballots.  Always nine ballots: stopping at
+// the digit's width through a run-time bound made the loop slower, not faster.
 __device__ __forceinline__ uint32_t same_value_lanes(uint32_t d) {
     uint32_t peers = 0xffffffffu;
 #pragma unroll
@@ -220,7 +223,7 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
     for (int i = 0; i < kSortIpt; ++i) {
         const int li = w * (32 * kSortIpt) + i * 32 + lane;
         const uint32_t d = li < tile_n ? ((uint32_t)(key[i] >> shift) & mask) : (uint32_t)kRadix;
-        const uint32_t peers = __match_any_sync(0xffffffffu, d);
+        const uint32_t peers = same_value_lanes(d);
         const int leader = __ffs(peers) - 1;
         uint32_t b = 0;
         if (lane == leader) { b = mycnt[d]; mycnt[d] = b + (uint32_t)__popc(peers); }
