@@ -10,6 +10,9 @@
 // twice: a symbolic pass that only counts (row lengths -> positions by a scan -> sizes of C's
 // arrays, read back once), and a numeric pass that fills coordinates and values.
 // Cost per row is proportional to its products plus dims[1]/32 bitmap words.
+// When a dense row of C and its bitmap fit in shared memory (dims[1] up to about 25,000) the
+// workspace lives there and the expansion's atomics never leave the SM; wider results use one
+// workspace row per block in global memory (L2-resident).
 #include "common.cuh"
 
 namespace {
@@ -40,7 +43,7 @@ __device__ __forceinline__ uint32_t block_excl_scan_u32(uint32_t v, uint32_t* su
 
 // NUMERIC = false: rowlen[i] = number of distinct columns of row i.
 // NUMERIC = true : crd / val of C filled at cpos[i].. ; the workspace row is left zeroed.
-template <typename P, typename I, bool NUMERIC>
+template <typename P, typename I, bool NUMERIC, bool SMEM>
 __global__ void __launch_bounds__(kPThreads)
 k_spmspm(const P* __restrict__ apos, const I* __restrict__ acrd, const double* __restrict__ aval,
          const P* __restrict__ bpos, const I* __restrict__ bcrd, const double* __restrict__ bval, int64_t m,
@@ -50,8 +53,20 @@ k_spmspm(const P* __restrict__ apos, const I* __restrict__ acrd, const double* _
     __shared__ uint32_t sums[kPThreads / 32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int64_t words = (n + 31) >> 5;
-    double* ws = ws_all + (int64_t)blockIdx.x * n;            // this block's dense row of C
-    uint32_t* bm = bm_all + (int64_t)blockIdx.x * words;      // ... and its "filled" flags, one bit per column
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    double* ws;          // this block's dense row of C
+    uint32_t* bm;        // ... and its "filled" flags, one bit per column
+    if (SMEM) {          // [bitmap words, padded to 8 bytes][row of C, numeric pass only]; both start zeroed
+        bm = reinterpret_cast<uint32_t*>(s_dyn);
+        ws = reinterpret_cast<double*>(s_dyn + ((words * 4 + 7) & ~(int64_t)7));
+        for (int64_t x = threadIdx.x; x < words; x += kPThreads) bm[x] = 0u;
+        if (NUMERIC)
+            for (int64_t x = threadIdx.x; x < n; x += kPThreads) ws[x] = 0.0;
+        __syncthreads();
+    } else {
+        ws = ws_all + (int64_t)blockIdx.x * n;
+        bm = bm_all + (int64_t)blockIdx.x * words;
+    }
 
     for (int64_t i = blockIdx.x; i < m; i += gridDim.x) {
         // expand: every product of row i lands in the workspace
@@ -150,17 +165,39 @@ extern "C" sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBi
     const int64_t m = A->dims[0], n = B->dims[1];
     if (n > 0 && (uint64_t)(n - 1) > sp_width_max(crdBits)) return SP_ERR_WIDTH_OVERFLOW;
 
+    const int64_t words = (n + 31) >> 5;
+    // shared-memory workspace if one row of C and its bitmap fit next to a second block's
+    int dev = 0, sms = 0, smem_max = 0;
+    SP_CUDA(cudaGetDevice(&dev));
+    SP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    SP_CUDA(cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    const size_t shm_sym = (size_t)((words * 4 + 7) & ~(int64_t)7);
+    const size_t shm_num = shm_sym + (size_t)n * sizeof(double);
+    const bool in_smem = shm_num + 2048 <= (size_t)smem_max;
+    auto blocks_for = [&](size_t shm) {
+        int64_t per_sm = (int64_t)((size_t)smem_max / (shm + 1024));
+        if (per_sm > 8) per_sm = 8;
+        if (per_sm < 1) per_sm = 1;
+        int64_t b = per_sm * sms;
+        if (b > m) b = m;
+        return b < 1 ? (int64_t)1 : b;
+    };
     int64_t nblocks = m < 148 * 4 ? m : 148 * 4;
     if (nblocks < 1) nblocks = 1;
-    const int64_t words = (n + 31) >> 5;
     sp_workspace ws(stream);
-    double* wsrow = ws.get<double>((size_t)nblocks * n);
-    uint32_t* bm = ws.get<uint32_t>((size_t)nblocks * words);
+    double* wsrow = nullptr;
+    uint32_t* bm = nullptr;
+    if (!in_smem) {
+        wsrow = ws.get<double>((size_t)nblocks * n);
+        bm = ws.get<uint32_t>((size_t)nblocks * words);
+    }
     int64_t* rowlen = ws.get<int64_t>((size_t)m + 1);
     int64_t* d_count = ws.get<int64_t>(1);
     if (ws.failed) return SP_ERR_ALLOC;
-    SP_CUDA(cudaMemsetAsync(wsrow, 0, (size_t)nblocks * n * sizeof(double), stream));
-    SP_CUDA(cudaMemsetAsync(bm, 0, (size_t)nblocks * words * sizeof(uint32_t), stream));
+    if (!in_smem) {
+        SP_CUDA(cudaMemsetAsync(wsrow, 0, (size_t)nblocks * n * sizeof(double), stream));
+        SP_CUDA(cudaMemsetAsync(bm, 0, (size_t)nblocks * words * sizeof(uint32_t), stream));
+    }
 
     sp_tensor* C = new sp_tensor();
     cudaGetDevice(&C->device);
@@ -174,12 +211,20 @@ extern "C" sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBi
     if (!C->pos[1]) { sp_free(C); return SP_ERR_ALLOC; }
     auto fail = [&](sp_status s) { sp_free(C); return s; };
 
+#define SP_SPMSPM_ARGS                                                                                            \
+    static_cast<const P*>(A->pos[1]), static_cast<const I*>(A->crd[1]), A->val, static_cast<const P*>(B->pos[1]), \
+        static_cast<const I*>(B->crd[1]), B->val, m, n, wsrow, bm, rowlen, C->pos[1], posBits, C->crd[1], crdBits, C->val
 #define SP_SPMSPM_LAUNCH(NUM)                                                                                     \
     SP_DISPATCH_WIDTHS(A, {                                                                                       \
-        k_spmspm<P, I, NUM><<<(unsigned)nblocks, kPThreads, 0, stream>>>(                                         \
-            static_cast<const P*>(A->pos[1]), static_cast<const I*>(A->crd[1]), A->val,                           \
-            static_cast<const P*>(B->pos[1]), static_cast<const I*>(B->crd[1]), B->val, m, n, wsrow, bm, rowlen,  \
-            C->pos[1], posBits, C->crd[1], crdBits, C->val);                                          \
+        if (in_smem) {                                                                                            \
+            const size_t shm = NUM ? shm_num : shm_sym;                                                           \
+            if (cudaFuncSetAttribute(k_spmspm<P, I, NUM, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                                     (int)shm) != cudaSuccess)                                                    \
+                return fail(SP_ERR_CUDA);                                                                         \
+            k_spmspm<P, I, NUM, true><<<(unsigned)blocks_for(shm), kPThreads, shm, stream>>>(SP_SPMSPM_ARGS);     \
+        } else {                                                                                                  \
+            k_spmspm<P, I, NUM, false><<<(unsigned)nblocks, kPThreads, 0, stream>>>(SP_SPMSPM_ARGS);              \
+        }                                                                                                         \
     })
     if (m > 0) SP_SPMSPM_LAUNCH(false);
     k_row_offsets<<<1, kPThreads, 0, stream>>>(rowlen, m, C->pos[1], posBits, d_count);
@@ -201,6 +246,7 @@ extern "C" sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBi
         sp_count_launches(1);
     }
 #undef SP_SPMSPM_LAUNCH
+#undef SP_SPMSPM_ARGS
     *out = C;
     return SP_OK;
 }

@@ -25,7 +25,9 @@ def _check(oracle, A, B, pb=32, cb=32, bits=32):
 
 
 @pytest.mark.parametrize("m,k,n,na,nb", [(9, 7, 8, 20, 25), (30, 30, 30, 90, 90), (5, 6, 4, 0, 10), (12, 3, 40, 36, 100),
-                                         (700, 300, 9000, 5000, 20000), (64, 64, 33, 4096, 64 * 33)])
+                                         (700, 300, 9000, 5000, 20000), (64, 64, 33, 4096, 64 * 33),
+                                         # a result row too wide for shared memory: the global workspace path
+                                         (300, 200, 60000, 3000, 30000), (40, 50, 28500, 600, 9000)])
 def test_small_and_ragged(oracle, m, k, n, na, nb):
     _check(oracle, I.uniform_matrix(m, k, na, seed=m), I.uniform_matrix(k, n, nb, seed=n + 1))
 
