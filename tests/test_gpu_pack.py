@@ -53,6 +53,26 @@ def test_matrices_spanning_tiles(oracle, m, n, nnz, enc):
     assert_storage_equal(t, ref)
 
 
+def test_widest_keys(oracle):
+    # the fused sort key holds at most 63 bits: 3 x 21 bits here (eight radix passes), 2 x 31 for the matrix;
+    # one bit more is refused, not truncated
+    dims = (1 << 21, 1 << 21, 1 << 21)
+    coo = I.uniform_tensor(dims, 9000, seed=12)
+    for od in [(0, 1, 2), (2, 0, 1)]:
+        t, ref = _pack_both(oracle, coo, (1, 1, 1), od, 32, 32, 32)
+        assert_storage_equal(t, ref)
+    mat = I.uniform_matrix(1 << 31, 1 << 31, 7000, seed=13)
+    for lt, od in [((1, 1), (0, 1)), ((1, 1), (1, 0))]:
+        t, ref = _pack_both(oracle, mat, lt, od, 64, 64, 64)
+        assert_storage_equal(t, ref)
+    b = sp()
+    big = I.Coo((1 << 22, 1 << 21, 1 << 21), [np.arange(10) * 7, np.arange(10) * 5, np.arange(10) * 3], np.ones(10))
+    coords, vals = to_dev(big, 32)
+    with pytest.raises(b.SpError) as e:
+        b.sp_pack(big.dims, coords, vals, (1, 1, 1))
+    assert e.value.code == 2
+
+
 def test_confined_rows_and_power_law(oracle):
     for coo in (I.config3(seed=1, n=1 << 14, nnz=60000), I.config2(seed=1, n=4096)):
         for lt, od in [((0, 1), (0, 1)), ((1, 1), (0, 1)), ((0, 1), (1, 0))]:
