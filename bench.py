@@ -95,6 +95,7 @@ def work_model(wl):
     k["mttkrp_csf"] = dict(flops=2 * R5 * (c5.nnz + F5), bytes=12 * c5.nnz + 2 * W * F5 + 8 * R5 * sum(c5.dims))
     # Dense rows the method fetches per stored entry (one row of the dense operand each; no reuse assumed):
     # rows fetched, doubles per row, rows of the table they are drawn from.
+    k["spmv_dcsr"]["gather"] = dict(rows=c3.nnz, row_elems=1, table_rows=n3)
     k["spmm_dcsr"]["gather"] = dict(rows=c3.nnz, row_elems=N3, table_rows=n3)
     k["spmm_csr"]["gather"] = dict(rows=c2.nnz, row_elems=N2, table_rows=c2.dims[1])
     k["sddmm_csr"]["gather"] = dict(rows=c4.nnz, row_elems=K4, table_rows=c4.dims[1])

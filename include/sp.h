@@ -297,7 +297,8 @@ sp_status sp_get_pack_profile(double* ms /* host */, int* npasses /* host, may b
  * up to a multiple of 8) rows each of a row-major table[rows x row_elems] (device,
  * 16-byte aligned, caller-owned) at pseudo-random row numbers derived from seed,
  * eight rows in flight per group, 16 bytes per lane per load.  row_elems is 16, 32,
- * 64 or 128 doubles (else SP_ERR_UNSUPPORTED).  sink (device, blocks*256 doubles)
+ * 64 or 128 doubles, or 1: then every lane fetches rows_per_group single 8-byte elements
+ * of its own (the access SpMV makes to x); anything else is SP_ERR_UNSUPPORTED.  sink (device, blocks*256 doubles)
  * receives per-thread sums so the loads cannot be dropped; *fetched (host, may be
  * NULL) receives the number of rows fetched, i.e. bytes moved = *fetched * row_elems * 8.
  *

@@ -46,6 +46,23 @@ k_probe_gather(const double* __restrict__ table, uint32_t rows, int64_t per_grou
     sink[t] = acc0 + acc1;
 }
 
+// Every lane fetches single 8-byte elements at uniformly random positions (what SpMV does with x).
+__global__ void __launch_bounds__(kPThreads)
+k_probe_gather_elems(const double* __restrict__ table, uint32_t n, int64_t per_lane, uint64_t seed,
+                     double* __restrict__ sink) {
+    const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    double acc = 0.0;
+    for (int64_t it = 0; it < per_lane; it += kInFlight) {
+        double v[kInFlight];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u)
+            v[u] = table[mix64(seed + (uint64_t)(t * per_lane + it + u) * 0x9E3779B97F4A7C15ull) % n];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) acc += v[u];
+    }
+    sink[t] = acc;
+}
+
 constexpr int kChains = 8;
 
 __global__ void __launch_bounds__(kPThreads)
@@ -73,6 +90,13 @@ extern "C" sp_status sp_probe_gather(const double* table, int64_t rows, int64_t 
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int64_t per = sp_ceil_div(rows_per_group, kInFlight) * kInFlight;
     int lpr = 0;
+    if (row_elems == 1) {      // single elements: one fetch per lane
+        k_probe_gather_elems<<<(unsigned)blocks, kPThreads, 0, stream>>>(table, (uint32_t)rows, per, seed, sink);
+        SP_LAUNCH_CHECK();
+        sp_count_launches(1);
+        if (fetched) *fetched = blocks * kPThreads * per;
+        return SP_OK;
+    }
     switch (row_elems) {
 #define SP_PROBE_CASE(E, LPR, NL)                                                                              \
     case E:                                                                                                    \

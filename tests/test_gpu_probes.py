@@ -15,7 +15,7 @@ def _ms(fn):
     return a.elapsed_time(b), n
 
 
-@pytest.mark.parametrize("row_elems,lanes", [(16, 8), (32, 8), (64, 16), (128, 32)])
+@pytest.mark.parametrize("row_elems,lanes", [(1, 1), (16, 8), (32, 8), (64, 16), (128, 32)])
 def test_gather_probe_counts_rows_and_moves_bytes(row_elems, lanes):
     table = torch.rand(4096, row_elems, dtype=torch.float64, device="cuda")
     blocks, per = 64, 100                      # 100 rounds up to 104 (a multiple of the 8 rows in flight)
