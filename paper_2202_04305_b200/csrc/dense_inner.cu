@@ -82,71 +82,138 @@ k_spmv_dense_cols(const double* __restrict__ val, const I* __restrict__ outer, i
     atomicAdd(y + i, s);
 }
 
-// SpMM with a dense inner level: C[i,:] = sum_k A[i,k] * B[k,:] where A's stored slices are dense.
-// A block owns kRT output rows and one 32-column tile of C and walks the contraction index in steps of
-// kKT: the kRT x kKT tile of A is staged in shared memory (stored [k][row], so a warp reads its four
-// row values with one 32-byte broadcast), each warp owns 4 rows, lane = column, and every B row is
-// loaded once per warp and used for 4 rows.
+// SpMM with a dense inner level: C[i,:] = sum_k A[i,k] * B[k,:] where A's stored slices are dense,
+// i.e. a plain f64 contraction - the one place on this path where tensor cores apply.  A block owns
+// a kRT x kCT tile of C and walks the contraction index in steps of kKT; each of its 8 warps owns
+// 32 rows x 32 columns as 4 x 4 tiles of the 8 x 8 x 4 f64 matrix instruction.  The kRT x kKT tile
+// of A (stored [k][row]) and the kKT x kCT tile of B sit in shared memory, double buffered: the
+// next tiles are fetched into registers before the current ones are used and written to the other
+// buffer afterwards, so one barrier per step suffices.  Operand fragments are one double per lane
+// (A: row lane/4, k lane%4; B: k lane%4, column lane/4), read with 8-byte shared loads; the row
+// strides are chosen so that the four k of a fragment fall on distinct banks.
 //   row-major    : output row = stored slice q (i = crd[0][q]), k = inner index,  A[q,k]  = val[q*inner + k]
 //   column-major : output row = inner index i,  k = stored slice q (crd[0][q]),   A[i,q]  = val[q*inner + i]
-constexpr int kRT = 32, kKT = 32;
+constexpr int kRT = 256, kKT = 8, kCT = 32;
+constexpr int kAStride = kRT + 4;               // doubles per k-row of the A tile: 520 words = 8 (mod 32 banks)
+constexpr int kBStride = kCT + 4;               // ... of the B tile: 72 words = 8 (mod 32)
+static_assert(kDThreads == kRT && kDThreads == kKT * kCT && kRT == 32 * (kDThreads / 32) && kCT == 32, "tile/thread layout");
+
+__device__ __forceinline__ void dmma_8x8x4(double& c0, double& c1, double a, double b) {
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                 : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
+}
 
 template <typename I, bool ROWMAJOR>
-__global__ void __launch_bounds__(kDThreads)
+__global__ void __launch_bounds__(kDThreads, 2)
 k_spmm_dense_inner(const double* __restrict__ val, const I* __restrict__ outer, int64_t nslices, int64_t inner,
                    const double* __restrict__ B, int64_t N, int64_t ldb, double* __restrict__ C, int64_t ldc,
-                   int64_t kchunk) {
-    __shared__ double s_a[kKT][kRT + 4];
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+                   int64_t kchunk, int vec_a) {
+    __shared__ __align__(16) double s_a[2][kKT][kAStride];
+    __shared__ __align__(16) double s_b[2][kKT][kBStride];
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
     const int64_t nrows = ROWMAJOR ? nslices : inner;     // output rows this kernel produces
     const int64_t nk = ROWMAJOR ? inner : nslices;        // length of the contraction
-    const int64_t r0 = (int64_t)blockIdx.x * kRT;
-    const int64_t col = (int64_t)blockIdx.y * 32 + lane;
-    const bool on = col < N;
-    const double* Bc = B + (on ? col : (int64_t)blockIdx.y * 32);
-    double acc[4] = {0.0, 0.0, 0.0, 0.0};
+    const int64_t r0 = (int64_t)blockIdx.x * kRT, c0 = (int64_t)blockIdx.y * kCT;
     // blockIdx.z owns the contraction range [kbeg, kend); with more than one range the partial
     // products are added into C (zeroed by the caller) with atomics
     const int64_t kbeg = (int64_t)blockIdx.z * kchunk;
     const int64_t kend = kbeg + kchunk < nk ? kbeg + kchunk : nk;
-    for (int64_t k0 = kbeg; k0 < kend; k0 += kKT) {
-        __syncthreads();
-        // stage A[r0 .. r0+kRT) x [k0 .. k0+kKT), zero outside
-        for (int e = threadIdx.x; e < kRT * kKT; e += kDThreads) {
-            // the fast index of the load follows the contiguous index of val
-            const int rr = ROWMAJOR ? e / kKT : e % kRT;
-            const int kk = ROWMAJOR ? e % kKT : e / kRT;
-            const int64_t r = r0 + rr, k = k0 + kk;
-            double a = 0.0;
-            if (r < nrows && k < kend) a = ROWMAJOR ? __ldcs(val + r * inner + k) : __ldcs(val + k * inner + r);
-            s_a[kk][rr] = a;
-        }
-        __syncthreads();
-        const int kmax = (int)(kend - k0 < kKT ? kend - k0 : kKT);
-        double b[kKT / 4];
-        for (int kb = 0; kb < kmax; kb += kKT / 4) {      // 8 B rows in flight per warp
+
+    // Loader roles.  Row-major with 16-byte aligned rows: four lanes cover the kKT values (64 bytes)
+    // of one row, a warp instruction covers 8 rows, a thread fetches a k-pair of 4 rows.
+    // Otherwise thread t fetches the kKT values of tile row t one by one (column-major: coalesced
+    // along the rows).  Every thread also fetches one element of the B tile.
+    double a_reg[kKT], b_reg;
+    const bool quad = ROWMAJOR && vec_a;
+    const int bk = t / kCT, bc = t % kCT;
+    auto load_tile = [&](int64_t k0) {
+        if (quad && k0 + kKT <= kend) {
 #pragma unroll
-            for (int u = 0; u < kKT / 4; ++u) {
-                const int64_t k = k0 + kb + u;
-                const int64_t krow = k < nk ? (ROWMAJOR ? k : (outer ? (int64_t)outer[k] : k)) : 0;
-                b[u] = __ldg(Bc + krow * ldb);
+            for (int j = 0; j < 4; ++j) {
+                const int64_t r = r0 + w * 32 + j * 8 + (lane >> 2);
+                double2 v = make_double2(0.0, 0.0);
+                if (r < nrows) v = __ldcs(reinterpret_cast<const double2*>(val + r * inner + k0) + (lane & 3));
+                a_reg[2 * j] = v.x; a_reg[2 * j + 1] = v.y;
             }
+        } else if (quad) {                                     // ragged last step of the range
 #pragma unroll
-            for (int u = 0; u < kKT / 4; ++u) {
-                if (kb + u < kmax) {
+            for (int j = 0; j < 4; ++j) {
+                const int64_t r = r0 + w * 32 + j * 8 + (lane >> 2), k = k0 + 2 * (lane & 3);
+                a_reg[2 * j] = (r < nrows && k < kend) ? __ldg(val + r * inner + k) : 0.0;
+                a_reg[2 * j + 1] = (r < nrows && k + 1 < kend) ? __ldg(val + r * inner + k + 1) : 0.0;
+            }
+        } else {
+            const int64_t lr = r0 + t;
 #pragma unroll
-                    for (int r = 0; r < 4; ++r) acc[r] = fma(s_a[kb + u][4 * w + r], b[u], acc[r]);
-                }
+            for (int kk = 0; kk < kKT; ++kk) {
+                const int64_t k = k0 + kk;
+                a_reg[kk] = (lr < nrows && k < kend) ? (ROWMAJOR ? __ldg(val + lr * inner + k) : __ldcs(val + k * inner + lr)) : 0.0;
             }
         }
+        const int64_t k = k0 + bk, c = c0 + bc;
+        b_reg = 0.0;
+        if (k < kend && c < N) b_reg = __ldg(B + (ROWMAJOR ? k : (outer ? (int64_t)outer[k] : k)) * ldb + c);
+    };
+    auto store_tile = [&](int buf) {
+        if (quad) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int r = w * 32 + j * 8 + (lane >> 2), kk = 2 * (lane & 3);
+                s_a[buf][kk][r] = a_reg[2 * j];
+                s_a[buf][kk + 1][r] = a_reg[2 * j + 1];
+            }
+        } else {
+#pragma unroll
+            for (int kk = 0; kk < kKT; ++kk) s_a[buf][kk][t] = a_reg[kk];
+        }
+        s_b[buf][bk][bc] = b_reg;
+    };
+
+    double acc[4][4][2];                        // [row tile][column tile][the lane's two columns]
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { acc[i][j][0] = 0.0; acc[i][j][1] = 0.0; }
+
+    int buf = 0;
+    if (kbeg < kend) {
+        load_tile(kbeg);
+        store_tile(0);
     }
-    if (on) {
+    __syncthreads();
+    const int fk = lane & 3, fr = lane >> 2;    // this lane's k and row/column inside a fragment
+    for (int64_t k0 = kbeg; k0 < kend; k0 += kKT) {
+        const bool more = k0 + kKT < kend;
+        if (more) load_tile(k0 + kKT);
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int64_t row = r0 + 4 * w + r;
-            if (row < nrows) {
-                double* dst = C + (ROWMAJOR ? (outer ? (int64_t)outer[row] : row) : row) * ldc + col;
-                if (gridDim.z > 1) atomicAdd(dst, acc[r]); else *dst = acc[r];
+        for (int k4 = 0; k4 < kKT; k4 += 4) {
+            double a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = s_a[buf][k4 + fk][w * 32 + i * 8 + fr];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = s_b[buf][k4 + fk][j * 8 + fr];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) dmma_8x8x4(acc[i][j][0], acc[i][j][1], a[i], b[j]);
+        }
+        if (more) store_tile(buf ^ 1);
+        __syncthreads();
+        buf ^= 1;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int64_t row = r0 + w * 32 + i * 8 + fr;
+        if (row >= nrows) continue;
+        double* dst = C + (ROWMAJOR ? (outer ? (int64_t)outer[row] : row) : row) * ldc;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int64_t col = c0 + j * 8 + 2 * fk + h;
+                if (col < N) {
+                    if (gridDim.z > 1) atomicAdd(dst + col, acc[i][j][h]); else dst[col] = acc[i][j][h];
+                }
             }
         }
     }
@@ -204,12 +271,12 @@ sp_status sp_spmm_dense_inner(const sp_tensor* A, const double* B, int64_t N, in
     }
     const int64_t nrows = rowmajor ? nslices : inner;
     const int64_t nk = rowmajor ? inner : nslices;
-    const int64_t rb = sp_ceil_div(nrows, kRT), cb = sp_ceil_div(N, 32);
+    const int64_t rb = sp_ceil_div(nrows, kRT), cb = sp_ceil_div(N, kCT);
     // few row blocks and a long contraction (a row band): split the contraction so every SM has work
     int64_t ksplit = 1;
-    if (rb * cb < 4 * 148) {
-        ksplit = sp_ceil_div(4 * 148, rb * cb);
-        const int64_t most = sp_ceil_div(nk, 8 * kKT);
+    if (rb * cb < 2 * 148) {
+        ksplit = sp_ceil_div(2 * 148, rb * cb);
+        const int64_t most = sp_ceil_div(nk, 16 * kKT);
         if (ksplit > most) ksplit = most;
         if (ksplit > 65535) ksplit = 65535;
         if (ksplit < 1) ksplit = 1;
@@ -222,11 +289,13 @@ sp_status sp_spmm_dense_inner(const sp_tensor* A, const double* B, int64_t N, in
     }
     if (cb > 65535) return SP_ERR_UNSUPPORTED;
     dim3 grid((unsigned)rb, (unsigned)cb, (unsigned)(ksplit > 0 ? ksplit : 1));
+    // 16-byte loads along a stored row need every row to start on a 16-byte boundary
+    const int vec_a = (inner % 2 == 0 && reinterpret_cast<uintptr_t>(A->val) % 16 == 0) ? 1 : 0;
 #define SP_DENSE_MM(I)                                                                                                  \
     do {                                                                                                                \
         const I* outer = outer_c ? static_cast<const I*>(A->crd[0]) : nullptr;                                          \
-        if (rowmajor) k_spmm_dense_inner<I, true><<<grid, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, B, N, ldb, C, ldc, kchunk); \
-        else k_spmm_dense_inner<I, false><<<grid, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, B, N, ldb, C, ldc, kchunk);       \
+        if (rowmajor) k_spmm_dense_inner<I, true><<<grid, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, B, N, ldb, C, ldc, kchunk, vec_a); \
+        else k_spmm_dense_inner<I, false><<<grid, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, B, N, ldb, C, ldc, kchunk, vec_a);       \
     } while (0)
     if (A->crdBits == 32) SP_DENSE_MM(uint32_t); else SP_DENSE_MM(uint64_t);
 #undef SP_DENSE_MM
