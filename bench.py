@@ -155,6 +155,9 @@ class GpuSuite:
         self.xv4 = f64(self.S4.nval)
         self.Qa = sp.sp_pack(wl["q_a"].dims, i32(wl["q_a"]), dev(wl["q_a"].vals), (0, 1))
         self.Qb = sp.sp_pack(wl["q_b"].dims, i32(wl["q_b"]), dev(wl["q_b"].vals), (0, 1))
+        # SpMM over the row band stored (compressed, dense): a dense f64 contraction (timed on its own, not in the step)
+        self.B1c = torch.rand(wl["c1b"].dims[1], 32, dtype=torch.float64, device="cuda") * 2 - 1
+        self.C1c = f64(wl["c1b"].dims[0], 32)
         self.flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
         torch.cuda.synchronize()
 
@@ -202,6 +205,7 @@ class GpuSuite:
             "pack_csf": lambda: sp.sp_pack(wl["c5"].dims, self.c5, self.v5, (1, 1, 1)).free(),
             "mttkrp_csf": lambda: sp.sp_mttkrp(csf(), self.Bf, self.Cf, self.M5),
             "next_spmspm_csr": lambda: sp.sp_spmspm(self.Qa, self.Qb).free(),
+            "next_spmm_cdr": lambda: sp.sp_spmm(self.A1c, self.B1c, self.C1c),
         }
 
     def flush_l2(self):
@@ -450,6 +454,8 @@ def main():
                          "frac_of_8TBs": round(gbs / 8000.0, 4)}
         if "units" in m:
             kernels[name]["Mnnz_per_s"] = round(m["units"] / (med * 1e-3) / 1e6, 1)
+        if name == "next_spmm_cdr":     # a dense contraction: bounded by the f64 multiply-add rate
+            kernels[name]["frac_of_measured_f64_peak"] = round(m["flops"] / (med * 1e-3) / 1e12 / bounds["dfma_tflops"], 4)
         if "gather" in m:
             # second bound: the rows the method fetches (one per stored entry) at the probed random-row rate
             g = m["gather"]
