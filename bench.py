@@ -443,6 +443,8 @@ def main():
     model["next_spmspm_csr"] = dict(flops=2 * products, bytes=12 * (qa.nnz + qb.nnz + qc.nval) + 4 * 3 * (qa.dims[0] + 1),
                                     units=products)
     qc.free()
+    m1, n1 = wl["c1b"].dims
+    model["next_spmm_cdr"] = dict(flops=2 * 32 * wl["rows1b"] * n1, bytes=8 * wl["rows1b"] * n1 + 8 * 32 * (n1 + m1))
     bounds = secondary_bounds(sp, torch, model)
     for name, fn in calls.items():
         ts = suite.time_call(fn, args.kernel_reps)

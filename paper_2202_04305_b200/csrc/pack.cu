@@ -71,8 +71,11 @@ struct LevelPlan {
 // ------------------------------------------------------------------ keys ---
 struct LevelCoords { const void* p[SP_MAX_RANK]; };   // coordinate array of the dimension stored at level l
 
+// idx_bits > 0: the entry index rides in the low idx_bits bits of the key itself (the sort then
+// moves 8 bytes per entry instead of 12) and no index array is written.
 template <typename CT>
-__global__ void k_build_keys(LevelCoords lc, int64_t n, LevelPlan p, uint64_t* keys, uint32_t* idx, int* err) {
+__global__ void k_build_keys(LevelCoords lc, int64_t n, LevelPlan p, uint64_t* keys, uint32_t* idx, int idx_bits,
+                             int* err) {
     int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (e >= n) return;
     uint64_t key = 0;
@@ -86,8 +89,12 @@ __global__ void k_build_keys(LevelCoords lc, int64_t n, LevelPlan p, uint64_t* k
         }
     }
     if (bad) atomicOr(err, kErrRange);
-    keys[e] = key;
-    idx[e] = (uint32_t)e;
+    if (idx_bits > 0) {
+        keys[e] = (key << idx_bits) | (uint64_t)e;
+    } else {
+        keys[e] = key;
+        idx[e] = (uint32_t)e;
+    }
 }
 
 // ------------------------------------------------------------ radix sort ---
@@ -184,18 +191,24 @@ k_sort_scan(uint32_t* tilehist, int64_t ntiles, uint32_t* digit_total) {
     if (threadIdx.x == 0) digit_total[blockIdx.x] = carry;
 }
 
-constexpr size_t kDownSmem = (size_t)kSortTile * 8 + (size_t)kSortTile * 4 +
-                             (size_t)kSortWarps * (kRadix + 1) * 4 + (size_t)(kRadix + 1) * 4 + (size_t)kRadix * 8 + 64;
+constexpr size_t down_smem(bool pay) {
+    return (size_t)kSortTile * 8 + (pay ? (size_t)kSortTile * 4 : 0) + (size_t)kSortWarps * (kRadix + 1) * 4 +
+           (size_t)(kRadix + 1) * 4 + (size_t)kRadix * 8 + 64;
+}
 
+// PAY: a 32-bit payload (the entry index) travels beside every key.  Without it the index sits in
+// the key's low bits; the last pass (split_bits >= 0) then separates the two again on the way out:
+// keys_out gets key >> split_bits, idx_out the low split_bits bits.
+template <bool PAY>
 __global__ void __launch_bounds__(kSortThreads, 3)   // three tiles per SM hide the ranking chain's latency
 k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict__ idx_in,
                  uint64_t* __restrict__ keys_out, uint32_t* __restrict__ idx_out, int64_t n, int shift,
                  uint32_t mask, const uint32_t* __restrict__ tilehist, int64_t ntiles,
-                 const uint32_t* __restrict__ digit_total) {
+                 const uint32_t* __restrict__ digit_total, int split_bits) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t* skeys = reinterpret_cast<uint64_t*>(smem_raw);
     uint32_t* sidx = reinterpret_cast<uint32_t*>(skeys + kSortTile);
-    uint32_t* wcnt = sidx + kSortTile;                       // [warps][kRadix + 1]
+    uint32_t* wcnt = PAY ? sidx + kSortTile : sidx;           // [warps][kRadix + 1]
     uint32_t* dstart = wcnt + kSortWarps * (kRadix + 1);      // [kRadix + 1]
     int64_t* goff = reinterpret_cast<int64_t*>(dstart + (kRadix + 1) + 1);   // [kRadix], 8-byte aligned
     __shared__ uint32_t sums[8];
@@ -217,7 +230,7 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
         const int li = w * (32 * kSortIpt) + i * 32 + lane;
         const bool valid = li < tile_n;
         key[i] = valid ? keys_in[base + li] : 0;
-        pay[i] = valid ? idx_in[base + li] : 0;
+        pay[i] = (PAY && valid) ? idx_in[base + li] : 0;
     }
 #pragma unroll
     for (int i = 0; i < kSortIpt; ++i) {
@@ -269,15 +282,25 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
         bool valid = li < tile_n;
         uint32_t d = valid ? ((uint32_t)(key[i] >> shift) & mask) : (uint32_t)kRadix;
         uint32_t s = dstart[d] + mycnt[d] + rank[i];
-        if (valid) { skeys[s] = key[i]; sidx[s] = pay[i]; }
+        if (valid) {
+            skeys[s] = key[i];
+            if (PAY) sidx[s] = pay[i];
+        }
     }
     __syncthreads();
     for (int s = t; s < tile_n; s += kSortThreads) {
         uint64_t k = skeys[s];
         uint32_t d = (uint32_t)(k >> shift) & mask;
         int64_t o = goff[d] + s;
-        keys_out[o] = k;
-        idx_out[o] = sidx[s];
+        if (PAY) {
+            keys_out[o] = k;
+            idx_out[o] = sidx[s];
+        } else if (split_bits >= 0) {
+            keys_out[o] = split_bits < 64 ? k >> split_bits : 0;
+            idx_out[o] = (uint32_t)(k & ((1ull << split_bits) - 1ull));
+        } else {
+            keys_out[o] = k;
+        }
     }
 }
 
@@ -680,26 +703,39 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
 
         LevelCoords lc;
         for (int l = 0; l < SP_MAX_RANK; ++l) lc.p[l] = coo_coords[l < rank ? plan.src[l] : 0];
+        const int npasses = (total_bits + 7) / 8;
+        // the entry index rides inside the key when both fit in 64 bits
+        int idx_bits = 0;
+        while (((int64_t)1 << idx_bits) < n) ++idx_bits;
+        const bool fused = npasses > 0 && idx_bits > 0 && total_bits + idx_bits <= 64;
         const unsigned kb = (unsigned)sp_ceil_div(n, 256);
-        if (coo_coord_bits == 32) k_build_keys<int32_t><<<kb, 256, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], d_err);
-        else k_build_keys<int64_t><<<kb, 256, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], d_err);
+        if (coo_coord_bits == 32)
+            k_build_keys<int32_t><<<kb, 256, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], fused ? idx_bits : 0, d_err);
+        else
+            k_build_keys<int64_t><<<kb, 256, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], fused ? idx_bits : 0, d_err);
         SP_LAUNCH_CHECK();
         sp_count_launches(1);
         timer.mark(kPhKeys);
-        SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDownSmem));
-        const int npasses = (total_bits + 7) / 8;
+        SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)down_smem(true)));
+        SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)down_smem(false)));
         const int per = npasses ? (total_bits + npasses - 1) / npasses : 0;
         int cur = 0;
         for (int ps = 0; ps < npasses; ++ps) {
-            const int shift = ps * per;
-            const int width = (shift + per <= total_bits) ? per : (total_bits - shift);
+            const int kshift = ps * per;                     // position of the digit inside the level key
+            const int width = (kshift + per <= total_bits) ? per : (total_bits - kshift);
+            const int shift = kshift + (fused ? idx_bits : 0);
             const uint32_t mask = (1u << width) - 1u;
             k_sort_upsweep<<<(unsigned)stiles, kSortThreads, 0, stream>>>(kbuf[cur], n, shift, mask, tilehist, stiles);
             timer.mark(kPhUpsweep);
             k_sort_scan<<<kRadix, 256, 0, stream>>>(tilehist, stiles, digit_total);
             timer.mark(kPhScan);
-            k_sort_downsweep<<<(unsigned)stiles, kSortThreads, kDownSmem, stream>>>(
-                kbuf[cur], ibuf[cur], kbuf[cur ^ 1], ibuf[cur ^ 1], n, shift, mask, tilehist, stiles, digit_total);
+            if (fused)
+                k_sort_downsweep<false><<<(unsigned)stiles, kSortThreads, down_smem(false), stream>>>(
+                    kbuf[cur], nullptr, kbuf[cur ^ 1], ibuf[cur ^ 1], n, shift, mask, tilehist, stiles, digit_total,
+                    ps == npasses - 1 ? idx_bits : -1);
+            else
+                k_sort_downsweep<true><<<(unsigned)stiles, kSortThreads, down_smem(true), stream>>>(
+                    kbuf[cur], ibuf[cur], kbuf[cur ^ 1], ibuf[cur ^ 1], n, shift, mask, tilehist, stiles, digit_total, -1);
             SP_LAUNCH_CHECK();
             timer.mark(kPhDownsweep);
             sp_count_launches(3);

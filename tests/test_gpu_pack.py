@@ -97,6 +97,12 @@ def test_duplicates_zeros_and_flags(oracle):
     for lt, od in [((0, 1), (0, 1)), ((1, 1), (1, 0)), ((1, 0), (0, 1))]:
         t, ref = _pack_both(oracle, dup, lt, od)
         assert_storage_equal(t, ref)          # same summation order => same bits
+    # the same with keys too wide to carry the entry index inside them (the index travels as a payload then)
+    wide = I.uniform_tensor((1 << 20, 1 << 20, 1 << 20), 3000, seed=9)
+    wc = [np.concatenate([c, c[:400], c[100:300]]) for c in wide.coords]
+    wv = np.concatenate([wide.vals, I.uniform_pm1(8, 71, 600)])
+    t, ref = _pack_both(oracle, I.Coo(wide.dims, wc, wv), (1, 1, 1), (1, 2, 0))
+    assert_storage_equal(t, ref)
     b = sp()
     c, v = to_dev(dup)
     with pytest.raises(b.SpError) as e:
