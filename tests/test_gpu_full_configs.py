@@ -115,6 +115,12 @@ def test_row_band_spmv(oracle):
     y = sp().sp_spmv(A, dev(x)).cpu().numpy()
     assert_close(y[rows], ref, bd, "row band CDR")
     assert np.all(y[1000:] == 0)
+    # SpMM over the same handle: the dense contraction (split over the inner dimension, summed with atomics)
+    B = I.dense_operand(0, 39, 65536, 32)
+    Cg = sp().sp_spmm(A, dev(B)).cpu().numpy()
+    cref, cbd = oracle.spmm(65536, coo.coords[0], coo.coords[1], coo.vals, B, rows)
+    assert_close(Cg[rows], cref, cbd, "row band CDR SpMM")
+    assert np.all(Cg[1000:] == 0)
     for lt in [(0, 1), (1, 1)]:
         A = sp().sp_pack(coo.dims, coords, vals, lt)
         y = sp().sp_spmv(A, dev(x)).cpu().numpy()
