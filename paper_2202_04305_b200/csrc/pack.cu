@@ -367,13 +367,13 @@ k_count_flags(const uint64_t* __restrict__ keys, int64_t n, LevelPlan p, uint64_
 
 static_assert(kField * SP_MAX_RANK <= 64 && (1 << kField) > kCtTile, "packed per-tile counters");
 
-// Single block (512 threads): tilesum (packed) -> tileprefix[l][tile] (exclusive), counts[l].
+// One block (512 threads) per level: tilesum (packed) -> tileprefix[l][tile] (exclusive), counts[l].
 // Across tiles the counts outgrow the packed fields, so each level is scanned on its own.
 __global__ void __launch_bounds__(512)
 k_scan_tiles(const uint64_t* __restrict__ tilesum, int64_t ntiles, int rank, int64_t* __restrict__ tileprefix,
              int64_t* __restrict__ counts) {
     __shared__ uint64_t sums[16];
-    for (int l = 0; l < rank; ++l) {
+    for (int l = blockIdx.x; l < rank; l += gridDim.x) {
         uint64_t run = 0;
         for (int64_t base = 0; base < ntiles; base += 512) {
             const int64_t i = base + threadIdx.x;
@@ -746,7 +746,7 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
         idx = ibuf[cur];
 
         k_count_flags<<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum);
-        k_scan_tiles<<<1, 512, 0, stream>>>(tilesum, ct_tiles, rank, tileprefix, d_counts);
+        k_scan_tiles<<<rank, 512, 0, stream>>>(tilesum, ct_tiles, rank, tileprefix, d_counts);
         SP_LAUNCH_CHECK();
         timer.mark(kPhCount);
         sp_count_launches(3);
