@@ -90,19 +90,34 @@ k_spmspm(const P* __restrict__ apos, const I* __restrict__ acrd, const double* _
             uint32_t bits = wi < words ? bm[wi] : 0u;
             uint32_t tot;
             const uint32_t ex = block_excl_scan_u32((uint32_t)__popc(bits), sums, &tot);
-            if (wi < words && bits) {
-                bm[wi] = 0u;
-                if (NUMERIC) {
-                    int64_t slot = base + carry + ex;
-                    while (bits) {
-                        const int bpos_ = __ffs(bits) - 1;
-                        bits &= bits - 1;
-                        const int64_t j = (wi << 5) + bpos_;
+            if (wi < words && bits) bm[wi] = 0u;
+            if (NUMERIC && tot >= 8u * kPThreads) {
+                // well-filled words: a warp empties its 32 words one after the other, lane = bit, so the
+                // workspace row is read (and cleared) 32 adjacent columns at a time and C is written in order
+                const uint32_t below = (1u << lane) - 1u;
+                for (uint32_t todo = __ballot_sync(0xffffffffu, bits != 0u); todo; todo &= todo - 1u) {
+                    const int q = __ffs(todo) - 1;                      // next word of this warp that has columns
+                    const uint32_t wbits = __shfl_sync(0xffffffffu, bits, q);
+                    const uint32_t woff = __shfl_sync(0xffffffffu, ex, q);
+                    if ((wbits >> lane) & 1u) {
+                        const int64_t j = ((w0 + (int64_t)(w * 32 + q)) << 5) + lane;
+                        const int64_t slot = base + carry + woff + __popc(wbits & below);
                         sp_store_uint(ccrd, slot, (uint64_t)j, ccrdBits);
                         cval[slot] = ws[j];
                         ws[j] = 0.0;
-                        ++slot;
                     }
+                }
+            } else if (NUMERIC && wi < words && bits) {
+                // sparse words: every thread walks the few columns of its own word
+                int64_t slot = base + carry + ex;
+                while (bits) {
+                    const int bpos_ = __ffs(bits) - 1;
+                    bits &= bits - 1;
+                    const int64_t j = (wi << 5) + bpos_;
+                    sp_store_uint(ccrd, slot, (uint64_t)j, ccrdBits);
+                    cval[slot] = ws[j];
+                    ws[j] = 0.0;
+                    ++slot;
                 }
             }
             carry += tot;
