@@ -168,6 +168,9 @@ sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* stream);
  * (Sections 1 and 5.2).  B is dims[1] x N with leading dimension ldb, C is
  * dims[0] x N with ldc.  Encodings (all eight two-dimensional ones, the set the
  * search loop of Section 5.2 enumerates) and the atomics remark as for sp_spmv.
+ * With a dense inner level the product is a dense contraction; when it has few
+ * output rows its contraction index is split over thread blocks and the partial
+ * sums meet in C through atomics too (row-major included).
  */
 sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t ldb,
                   double* C, int64_t ldc, void* stream);
