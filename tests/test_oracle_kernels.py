@@ -115,6 +115,21 @@ def test_mttkrp_ones_counts_slice_entries(oracle):
     assert np.array_equal(M, np.repeat(np.bincount(coo.coords[0], minlength=6)[:, None], 3, 1))
 
 
+def test_mttkrp_row_sampling_equals_full(oracle):
+    t = I.uniform_tensor((9, 7, 6), 120, seed=13)
+    R = 5
+    Bf = I.dense_operand(3, 53, t.dims[1], R)
+    Cf = I.dense_operand(3, 54, t.dims[2], R)
+    full, fb = oracle.mttkrp(t.dims[0], *t.coords, t.vals, Bf, Cf)
+    rows = np.array([t.dims[0] - 1, 0, 3, 5])
+    part, pb = oracle.mttkrp(t.dims[0], *t.coords, t.vals, Bf, Cf, rows)
+    assert np.array_equal(part, full[rows]) and np.array_equal(pb, fb[rows])
+    # and against the dense definition, so that a slot mapped to the wrong row cannot pass
+    T = np.zeros(t.dims)
+    T[t.coords[0], t.coords[1], t.coords[2]] = t.vals
+    assert np.allclose(part, np.einsum("ijk,jr,kr->ir", T, Bf, Cf)[rows], rtol=0, atol=1e-12)
+
+
 def test_exact_integer_inputs_are_exact(oracle):
     coo = I.uniform_matrix(20, 20, 120, seed=4, integer_values=True)
     B = I.dense_operand(6, 57, 20, 7, integer_values=True)
