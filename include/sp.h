@@ -27,14 +27,20 @@
  *   - Every call returns an sp_status; nothing throws across the boundary.
  *     An encoding a kernel does not handle yields SP_ERR_UNSUPPORTED, never a
  *     different algorithm on the host.
- *   - A handle is immutable after sp_pack.  Kernels cache work-partition tables
- *     inside it on first use; use a handle from one stream at a time.
+ *   - A handle is immutable after sp_pack.  Kernels cache read-only work-partition
+ *     tables inside it on first use (under the handle's lock; a call on another
+ *     stream waits for the stream that built them); everything a call writes
+ *     besides its output is scratch it takes from the allocator for that call, so
+ *     calls on different streams or host threads may share a handle.  The handle
+ *     must be used with the device it was packed on current
+ *     (SP_ERR_INVALID_ARG otherwise).
  *   - CUDA graphs: once a kernel call has run on a handle (so its cached tables
  *     exist), later sp_spmv / sp_spmm / sp_sddmm / sp_mttkrp calls on it only
- *     enqueue stream-ordered work and may be stream-captured, provided the
- *     installed allocator is itself legal during capture (a stream-ordered or
- *     caching pool; the default cudaMalloc is not).  sp_pack, sp_convert, sp_unpack
- *     and sp_spmspm read sizes back to the host and cannot be captured.
+ *     enqueue stream-ordered work (kernels, memsets and allocator calls for
+ *     their scratch) and may be stream-captured, provided the installed
+ *     allocator is itself legal during capture (a stream-ordered or caching
+ *     pool).  sp_pack, sp_convert, sp_unpack and sp_spmspm read sizes back to
+ *     the host and cannot be captured.
  */
 #ifndef SP_H
 #define SP_H
@@ -61,7 +67,8 @@ typedef enum {
     SP_ERR_DUPLICATE = 5,       /* SP_DUP_ERROR was set and two entries share coordinates */
     SP_ERR_ALLOC = 6,           /* the allocator returned NULL */
     SP_ERR_CUDA = 7,            /* a CUDA runtime call failed */
-    SP_ERR_TIMEOUT = 8,         /* a bounded device-side wait ran out */
+    SP_ERR_TIMEOUT = 8,         /* reserved (a bounded device-side wait ran out): no kernel here waits on
+                                   another, so no call returns it */
     SP_ERR_TOO_LARGE = 9        /* the problem does not fit a fixed-capacity entry point (sp_spmv_static) */
 } sp_status;
 
@@ -74,8 +81,10 @@ const char* sp_status_string(sp_status s);
 /*
  * Workspace and storage allocator.  alloc(bytes, stream, ctx) returns device
  * memory usable on `stream`; dealloc returns it.  Both NULL restores the
- * default (cudaMalloc / cudaFree).  Process-wide; set it before the first
- * sp_pack and do not change it while handles are alive.
+ * default (the device's stream-ordered pool: cudaMallocAsync / cudaFreeAsync).
+ * Process-wide; set it before the first sp_pack and do not change it while
+ * handles are alive.  When alloc returns NULL the call in progress gives back
+ * everything it had taken and returns SP_ERR_ALLOC.
  */
 sp_status sp_set_allocator(void* (*alloc)(size_t bytes, void* stream, void* ctx),
                            void (*dealloc)(void* ptr, void* stream, void* ctx), void* ctx);
@@ -168,9 +177,12 @@ sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* stream);
  * (Sections 1 and 5.2).  B is dims[1] x N with leading dimension ldb, C is
  * dims[0] x N with ldc.  Encodings (all eight two-dimensional ones, the set the
  * search loop of Section 5.2 enumerates) and the atomics remark as for sp_spmv.
- * With a dense inner level the product is a dense contraction; when it has few
- * output rows its contraction index is split over thread blocks and the partial
- * sums meet in C through atomics too (row-major included).
+ * With a dense inner level the product is a dense contraction and runs on the
+ * f64 matrix instruction (the one place in this library where tensor cores
+ * apply; the sparse kernels are gathers and use none); when it has few output
+ * rows its contraction index is split over thread blocks and the partial sums
+ * meet in C through atomics too (row-major included).  A column-major matrix
+ * with 2^32 or more columns is refused (SP_ERR_UNSUPPORTED).
  */
 sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t ldb,
                   double* C, int64_t ldc, void* stream);
@@ -249,8 +261,8 @@ sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBits, int crd
  * living inside a host application that owns the GPU heap and forbids foreign
  * allocations, or a service whose allocator may block or fail under memory
  * pressure at exactly the moment the product is needed.  sp_spmv obtains its
- * work-partition table and row-carry buffer through the allocator on a handle's
- * first use; this call never does.  It calls neither the installed allocator nor
+ * work-partition table (on a handle's first use) and its row-carry buffer (on
+ * every call) through the allocator; this call never does.  It calls neither the installed allocator nor
  * cudaMalloc / cudaFree, and caches nothing in the handle.
  *
  * Its scratch is a fixed array compiled into the library (about 2 MiB of device
@@ -276,42 +288,10 @@ sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBits, int crd
 sp_status sp_spmv_static(const sp_tensor* A, const double* x, double* y, void* stream);
 
 /*
- * Measurement aids (no counterpart in the paper).
- * sp_launch_count: number of kernels this library has launched in this process.
- * sp_set_profiling(1): sp_pack brackets its phases with CUDA events on the caller's
- * stream (this adds small gaps between its kernels; leave it off when timing calls).
- * sp_get_pack_profile: milliseconds of the last profiled sp_pack per phase
- * (ms has SP_PACK_PROFILE_LEN entries: key build, sort histograms, sort scans,
- * sort scatters, node counting, emit + fill) and the number of sort passes.
+ * sp_launch_count: number of kernels this library has launched in this process (no
+ * counterpart in the paper; lets a caller check that work ran on the device).
  */
-#define SP_PACK_PROFILE_LEN 6
 int64_t sp_launch_count(void);
-sp_status sp_set_profiling(int enabled);
-sp_status sp_get_pack_profile(double* ms /* host */, int* npasses /* host, may be NULL */);
-
-/*
- * Probes of the two secondary bounds of the gather kernels (no counterpart in the
- * paper): SpMM, SDDMM and MTTKRP fetch one dense row per stored entry, so besides
- * HBM they are limited by the rate at which SMs can pull randomly chosen rows of a
- * cache-resident table, and by the f64 multiply-add rate.  Both calls enqueue one
- * kernel on stream and return at once; the caller times them with events.
- *
- * sp_probe_gather: blocks x 256 threads; lane groups fetch rows_per_group (rounded
- * up to a multiple of 8) rows each of a row-major table[rows x row_elems] (device,
- * 16-byte aligned, caller-owned) at pseudo-random row numbers derived from seed,
- * eight rows in flight per group, 16 bytes per lane per load.  row_elems is 16, 32,
- * 64 or 128 doubles, or 1: then every lane fetches rows_per_group single 8-byte elements
- * of its own (the access SpMV makes to x); anything else is SP_ERR_UNSUPPORTED.  sink (device, blocks*256 doubles)
- * receives per-thread sums so the loads cannot be dropped; *fetched (host, may be
- * NULL) receives the number of rows fetched, i.e. bytes moved = *fetched * row_elems * 8.
- *
- * sp_probe_dfma: blocks x 256 threads each run eight independent chains of iters
- * dependent f64 fused multiply-adds held in registers; *fmas (host, may be NULL)
- * receives the total count (flops = 2 * *fmas).  sink as above.
- */
-sp_status sp_probe_gather(const double* table, int64_t rows, int64_t row_elems, int64_t blocks,
-                          int64_t rows_per_group, uint64_t seed, double* sink, int64_t* fetched, void* stream);
-sp_status sp_probe_dfma(int64_t blocks, int64_t iters, double* sink, int64_t* fmas, void* stream);
 
 #ifdef __cplusplus
 }

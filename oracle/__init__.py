@@ -199,3 +199,56 @@ def vec_dot(ai, av, bi, bv):
     bd = C.c_double()
     x = f(C.c_int64(av.size), _ptr(ai), _ptr(av, _PD), C.c_int64(bv.size), _ptr(bi), _ptr(bv, _PD), C.byref(bd))
     return float(x), float(bd.value)
+
+
+# ---------------------------------------------------------------------------
+# The same products as loop nests over packed storage, outer loop on all host cores
+# (the "N cores" leg of the CPU baseline).  s: a Storage from pack().  Each returns
+# (result, threads used).
+# ---------------------------------------------------------------------------
+def _rowmajor_matrix(s: Storage):
+    if len(s.dims) != 2 or s.ord != (0, 1) or s.lt[1] != COMPRESSED:
+        raise ValueError("row-major (dense|compressed, compressed) storage expected")
+    rowid = _i64(s.crd[0]) if s.lt[0] == COMPRESSED else None
+    pos1, crd1 = _i64(s.pos[1]), _i64(s.crd[1])
+    return rowid, pos1, crd1, pos1.size - 1
+
+
+def par_spmm(s: Storage, B):
+    B = _f64(B)
+    N = B.shape[1]
+    rowid, pos1, crd1, nstored = _rowmajor_matrix(s)
+    Cm = np.zeros((s.dims[0], N))
+    v = _f64(s.val)
+    nt = lib().orc_par_spmm(C.c_int64(nstored), _ptr(rowid) if rowid is not None else None, _ptr(pos1), _ptr(crd1),
+                            _ptr(v, _PD), _ptr(B, _PD), C.c_int64(N), C.c_int64(N), _ptr(Cm, _PD), C.c_int64(N))
+    return Cm, nt
+
+
+def par_spmv(s: Storage, x):
+    y, nt = par_spmm(s, _f64(x).reshape(-1, 1))
+    return y[:, 0], nt
+
+
+def par_sddmm(s: Storage, A, B):
+    A, B = _f64(A), _f64(B)
+    rowid, pos1, crd1, nstored = _rowmajor_matrix(s)
+    v = _f64(s.val)
+    x = np.zeros(v.size)
+    nt = lib().orc_par_sddmm(C.c_int64(nstored), _ptr(rowid) if rowid is not None else None, _ptr(pos1), _ptr(crd1),
+                             _ptr(v, _PD), _ptr(A, _PD), C.c_int64(A.shape[1]), _ptr(B, _PD), C.c_int64(B.shape[1]),
+                             C.c_int64(A.shape[1]), _ptr(x, _PD))
+    return x, nt
+
+
+def par_mttkrp(s: Storage, B, Cf):
+    if len(s.dims) != 3 or s.ord != (0, 1, 2) or s.lt[1] != COMPRESSED or s.lt[2] != COMPRESSED:
+        raise ValueError("(dense|compressed, compressed, compressed) storage in identity order expected")
+    B, Cf = _f64(B), _f64(Cf)
+    R = B.shape[1]
+    crd0 = _i64(s.crd[0]) if s.lt[0] == COMPRESSED else None
+    pos1, crd1, pos2, crd2, v = _i64(s.pos[1]), _i64(s.crd[1]), _i64(s.pos[2]), _i64(s.crd[2]), _f64(s.val)
+    M = np.zeros((s.dims[0], R))
+    nt = lib().orc_par_mttkrp(C.c_int64(pos1.size - 1), _ptr(crd0) if crd0 is not None else None, _ptr(pos1), _ptr(crd1),
+                              _ptr(pos2), _ptr(crd2), _ptr(v, _PD), _ptr(B, _PD), _ptr(Cf, _PD), C.c_int64(R), _ptr(M, _PD))
+    return M, nt

@@ -18,6 +18,12 @@
  *     x87 extended precision, together with the per-entry bound sum |a*b|
  *     against which the f64 result of any summation order is judged.
  *
+ *   - orc_par_* are the same products written as the loop nests Section 4.3
+ *     derives over packed storage (outer loop over stored rows / slices, inner
+ *     loops over pos[l][p] .. pos[l][p+1]), with the outer loop split over all
+ *     host cores by OpenMP: the "oracle, N cores" leg of the CPU baseline.  They
+ *     are pinned by the coordinate-loop functions above them.
+ *
  * Readings where the paper is silent:
  *   - dimOrdering: result l of the affine map names the logical dimension
  *     stored at level l ("parity unpinned" by the paper for 3-cycles: all its
@@ -357,4 +363,91 @@ double orc_vec_dot(int64_t na, const int64_t *ai, const double *av, int64_t nb, 
     }
     if (bound) *bound = (double)bnd;
     return (double)acc;
+}
+
+/* ------------------------------------------------------------------------
+ * The same products as loop nests over packed storage, outer loop in parallel
+ * (OpenMP, static blocks of rows; rows are independent, so no atomics).
+ * rowid: crd[0] when level 0 is compressed (stored row q is row rowid[q]), NULL
+ * when it is dense (q is the row).  Outputs must be zero-filled by the caller
+ * for rows that store nothing.  Each returns the number of threads used.
+ * ---------------------------------------------------------------------- */
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static int threads_used(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* C[i,:] = sum_p val[p] * B[crd1[p],:] over p in pos1[q] .. pos1[q+1]  (Section 1's matmul, row-major A) */
+int orc_par_spmm(int64_t nstored, const int64_t *rowid, const int64_t *pos1, const int64_t *crd1,
+                 const double *val, const double *B, int64_t N, int64_t ldb, double *C, int64_t ldc)
+{
+#pragma omp parallel
+    {
+        long double *acc = malloc(sizeof(long double) * (size_t)(N + 1));
+#pragma omp for schedule(static)
+        for (int64_t q = 0; q < nstored; ++q) {
+            for (int64_t j = 0; j < N; ++j) acc[j] = 0.0L;
+            for (int64_t p = pos1[q]; p < pos1[q + 1]; ++p) {
+                const double *brow = B + crd1[p] * ldb;
+                for (int64_t j = 0; j < N; ++j) acc[j] += (long double)val[p] * (long double)brow[j];
+            }
+            double *crow = C + (rowid ? rowid[q] : q) * ldc;
+            for (int64_t j = 0; j < N; ++j) crow[j] = (double)acc[j];
+        }
+        free(acc);
+    }
+    return threads_used();
+}
+
+/* x[p] = S.val[p] * sum_k A[i,k] * B[k,crd1[p]] for the stored entries of row-major S (Section 6.2) */
+int orc_par_sddmm(int64_t nstored, const int64_t *rowid, const int64_t *pos1, const int64_t *crd1,
+                  const double *sval, const double *A, int64_t lda, const double *B, int64_t ldb, int64_t K,
+                  double *x)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t q = 0; q < nstored; ++q) {
+        const double *arow = A + (rowid ? rowid[q] : q) * lda;
+        for (int64_t p = pos1[q]; p < pos1[q + 1]; ++p) {
+            long double dot = 0.0L;
+            for (int64_t k = 0; k < K; ++k) dot += (long double)arow[k] * (long double)B[k * ldb + crd1[p]];
+            x[p] = (double)((long double)sval[p] * dot);
+        }
+    }
+    return threads_used();
+}
+
+/* M[i,:] = sum over fibres f of slice q, entries p of fibre f of val[p] * B[crd1[f],:] * C[crd2[p],:]
+   (Section 6.3 over all-compressed storage; the three scalars are multiplied per entry, as in the expression) */
+int orc_par_mttkrp(int64_t nslices, const int64_t *crd0, const int64_t *pos1, const int64_t *crd1,
+                   const int64_t *pos2, const int64_t *crd2, const double *val,
+                   const double *B, const double *Cf, int64_t R, double *M)
+{
+#pragma omp parallel
+    {
+        long double *acc = malloc(sizeof(long double) * (size_t)(R + 1));
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t q = 0; q < nslices; ++q) {
+            for (int64_t r = 0; r < R; ++r) acc[r] = 0.0L;
+            for (int64_t f = pos1[q]; f < pos1[q + 1]; ++f) {
+                const double *brow = B + crd1[f] * R;
+                for (int64_t p = pos2[f]; p < pos2[f + 1]; ++p) {
+                    const double *crow = Cf + crd2[p] * R;
+                    for (int64_t r = 0; r < R; ++r)
+                        acc[r] += (long double)val[p] * (long double)brow[r] * (long double)crow[r];
+                }
+            }
+            double *mrow = M + (crd0 ? crd0[q] : q) * R;
+            for (int64_t r = 0; r < R; ++r) mrow[r] = (double)acc[r];
+        }
+        free(acc);
+    }
+    return threads_used();
 }

@@ -20,8 +20,7 @@ _LIB_PATH = os.path.join(_HERE, "libsp.so")
 
 SYMBOLS = ["sp_status_string", "sp_set_allocator", "sp_pack", "sp_free", "sp_info", "sp_positions",
            "sp_coordinates", "sp_values", "sp_unpack", "sp_spmv", "sp_spmm", "sp_sddmm", "sp_mttkrp",
-           "sp_set_profiling", "sp_get_pack_profile", "sp_launch_count", "sp_spmv_static", "sp_mttkrp_mode", "sp_spmspm", "sp_convert", "sp_scale", "sp_vec_dot",
-           "sp_probe_gather", "sp_probe_dfma"]
+           "sp_launch_count", "sp_spmv_static", "sp_mttkrp_mode", "sp_spmspm", "sp_convert", "sp_scale", "sp_vec_dot"]
 SPMV_STATIC_MAX_ITEMS = 134217728
 
 
@@ -249,40 +248,6 @@ def sp_mttkrp(T: SpTensor, B, Cf, M=None):
 
 def sp_launch_count() -> int:
     return int(_lib.sp_launch_count())
-
-
-def sp_set_profiling(enabled: bool):
-    _check(_lib.sp_set_profiling(C.c_int(1 if enabled else 0)), "sp_set_profiling")
-
-
-def sp_probe_gather(table: torch.Tensor, blocks: int, rows_per_group: int, seed: int = 1) -> int:
-    """Enqueue the random row-gather probe over table (rows x 16|32|64|128 float64); returns rows fetched."""
-    _f64(table, "table")
-    sink = torch.empty(blocks * 256, dtype=torch.float64, device="cuda")
-    n = C.c_int64()
-    _check(_lib.sp_probe_gather(_dptr(table), C.c_int64(table.shape[0]), C.c_int64(table.shape[1]), C.c_int64(blocks),
-                                C.c_int64(rows_per_group), C.c_uint64(seed), _dptr(sink), C.byref(n), _stream()),
-           "sp_probe_gather")
-    return n.value
-
-
-def sp_probe_dfma(blocks: int, iters: int) -> int:
-    """Enqueue the register-only f64 multiply-add probe; returns the number of fused multiply-adds."""
-    sink = torch.empty(blocks * 256, dtype=torch.float64, device="cuda")
-    n = C.c_int64()
-    _check(_lib.sp_probe_dfma(C.c_int64(blocks), C.c_int64(iters), _dptr(sink), C.byref(n), _stream()), "sp_probe_dfma")
-    return n.value
-
-
-PACK_PHASES = ("keys", "sort_hist", "sort_scan", "sort_scatter", "count", "emit")
-
-
-def sp_get_pack_profile():
-    """(dict phase -> ms, number of sort passes) of the last sp_pack run with profiling on."""
-    ms = (C.c_double * len(PACK_PHASES))()
-    n = C.c_int()
-    _check(_lib.sp_get_pack_profile(ms, C.byref(n)), "sp_get_pack_profile")
-    return {k: ms[i] for i, k in enumerate(PACK_PHASES)}, n.value
 
 
 def sp_mttkrp_mode(T: SpTensor, mode: int, factors, M=None):

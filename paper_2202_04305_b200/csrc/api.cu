@@ -12,17 +12,38 @@ std::atomic<int64_t> g_launches{0};
 
 void sp_count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+// Default allocator: the device's stream-ordered pool, so that the per-call scratch of the compute
+// calls costs neither a device synchronisation nor a trip to the driver's heap.
 void* sp_dev_alloc(size_t bytes, cudaStream_t stream) {
     if (g_alloc) return g_alloc(bytes, stream, g_ctx);
     void* p = nullptr;
-    if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (cudaMallocAsync(&p, bytes, stream) != cudaSuccess) { cudaGetLastError(); return nullptr; }
     return p;
 }
 
+// stream == nullptr (sp_free): release after everything enqueued so far has finished.
 void sp_dev_free(void* p, cudaStream_t stream) {
     if (!p) return;
     if (g_dealloc) { g_dealloc(p, stream, g_ctx); return; }
-    cudaFree(p);
+    if (stream) cudaFreeAsync(p, stream); else cudaFree(p);
+}
+
+sp_status sp_check_device(const sp_tensor* t) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SP_ERR_CUDA;
+    return dev == t->device ? SP_OK : SP_ERR_INVALID_ARG;
+}
+
+sp_status sp_partition_built(sp_partition* p, cudaStream_t stream) {
+    SP_CUDA(cudaEventCreateWithFlags(&p->ready, cudaEventDisableTiming));
+    SP_CUDA(cudaEventRecord(p->ready, stream));
+    p->built_on = stream;
+    return SP_OK;
+}
+
+sp_status sp_partition_wait(const sp_partition& p, cudaStream_t stream) {
+    if (p.ready && stream != p.built_on) SP_CUDA(cudaStreamWaitEvent(stream, p.ready, 0));
+    return SP_OK;
 }
 
 extern "C" {
@@ -39,7 +60,7 @@ const char* sp_status_string(sp_status s) {
         case SP_ERR_DUPLICATE: return "duplicate coordinates";
         case SP_ERR_ALLOC: return "device allocation failed";
         case SP_ERR_CUDA: return "CUDA runtime error";
-        case SP_ERR_TIMEOUT: return "bounded device-side wait ran out";
+        case SP_ERR_TIMEOUT: return "bounded device-side wait ran out (reserved: no call returns it)";
         case SP_ERR_TOO_LARGE: return "problem exceeds the fixed scratch capacity of this entry point";
     }
     return "unknown status";
@@ -64,11 +85,12 @@ sp_status sp_free(sp_tensor* t) {
     }
     if (t->owns_val) sp_dev_free(t->val, nullptr);
     if (t->wide) sp_free(t->wide);
+    if (t->wide_ready) cudaEventDestroy(t->wide_ready);
     for (auto& kv : t->parts) {
         sp_dev_free(kv.second.row, nullptr);
         sp_dev_free(kv.second.nz, nullptr);
         sp_dev_free(kv.second.aux, nullptr);
-        sp_dev_free(kv.second.carry, nullptr);
+        if (kv.second.ready) cudaEventDestroy(kv.second.ready);
     }
     delete t;
     cudaSetDevice(prev);

@@ -15,14 +15,18 @@
 // ---------------------------------------------------------------------------
 
 // Work-partition table cached in a handle: chunk w covers merge-path
-// coordinates [(row[w], nz[w]), (row[w+1], nz[w+1])).
+// coordinates [(row[w], nz[w]), (row[w+1], nz[w+1])).  The arrays are written once, by the
+// kernels enqueued on `built_on` when the table is created, and only read afterwards; `ready`
+// marks the end of that work so that a call on another stream can wait for it.  Scratch that a
+// call writes (row carries) is never kept here: every call takes its own from the allocator, so
+// calls on different streams share nothing writable.
 struct sp_partition {
     int64_t nchunks = 0;
     int64_t* row = nullptr;   // nchunks + 1 entries (device)
     int64_t* nz = nullptr;    // nchunks + 1 entries (device)
     int64_t* aux = nullptr;   // kernel-specific (MTTKRP: slice of each chunk start)
-    double* carry = nullptr;  // kernel-specific scratch sized by the creator
-    int64_t carry_elems = 0;
+    cudaEvent_t ready = nullptr;
+    cudaStream_t built_on = nullptr;
 };
 
 struct sp_tensor {
@@ -39,13 +43,22 @@ struct sp_tensor {
     int64_t nval = 0;
     int device = 0;
     std::mutex mu;
-    std::map<uint64_t, sp_partition> parts;   // key = (kind << 32) | items per chunk
+    std::map<uint64_t, sp_partition> parts;   // key = (kind << 56) | items per chunk
     // For handles stored with 8- or 16-bit positions/coordinates: a copy of the overhead arrays
     // widened to 32 bits that the compute kernels read (values shared, not copied).  Built on
     // first use by sp_widened(), owned by this handle.
     sp_tensor* wide = nullptr;
+    cudaEvent_t wide_ready = nullptr;
+    cudaStream_t wide_built_on = nullptr;
     bool owns_val = true;
 };
+
+// SP_ERR_INVALID_ARG unless the handle's arrays live on the current device.
+sp_status sp_check_device(const sp_tensor* t);
+// Marks the end of the work that fills a cached table (p->ready, p->built_on).
+sp_status sp_partition_built(sp_partition* p, cudaStream_t stream);
+// Makes `stream` wait for that work when it is not the stream that did it.
+sp_status sp_partition_wait(const sp_partition& p, cudaStream_t stream);
 
 // The handle the compute kernels should read: t itself when its widths are 32 or 64 bits,
 // otherwise its (cached) 32-bit shadow.
@@ -80,6 +93,15 @@ struct sp_workspace {
 };
 
 void sp_count_launches(int n);
+
+// One NVTX range per API call (visible in Nsight Systems / Compute timelines; a no-op costing a
+// few nanoseconds when no tool is attached).
+#include <nvtx3/nvToolsExt.h>
+struct sp_nvtx_range {
+    explicit sp_nvtx_range(const char* name) { nvtxRangePushA(name); }
+    ~sp_nvtx_range() { nvtxRangePop(); }
+};
+#define SP_API_RANGE(name) sp_nvtx_range nvtx_range__(name)
 
 #define SP_CUDA(call)                                   \
     do {                                                \
@@ -138,8 +160,7 @@ enum { SP_PART_MERGE_LAST = 1, SP_PART_MTTKRP = 2, SP_PART_SEGIDS = 3 };
 // For rank-2 (x, compressed) storage: the logical level-0 coordinate of every stored entry
 // (the expanded "outer" index), uint32, cached in the handle.  Needs dims < 2^32.
 sp_status sp_get_segment_ids(sp_tensor* t, cudaStream_t stream, const uint32_t** out);
-sp_status sp_get_merge_partition(sp_tensor* t, int64_t items_per_chunk, int64_t carry_elems_per_chunk,
-                                 cudaStream_t stream, sp_partition* out);
+sp_status sp_get_merge_partition(sp_tensor* t, int64_t items_per_chunk, cudaStream_t stream, sp_partition* out);
 sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t nnz_per_chunk, cudaStream_t stream, sp_partition* out);
 
 // SpMV for rank-2 handles whose inner level is dense (dense_inner.cu).

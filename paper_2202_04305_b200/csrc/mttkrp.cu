@@ -390,6 +390,7 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
 static sp_status mttkrp_levels(sp_tensor* T, const double* F1, const double* F2, int64_t R, double* M, cudaStream_t stream);
 
 extern "C" sp_status sp_mttkrp(sp_tensor* T, const double* B, const double* C, int64_t R, double* M, void* stream_) {
+    SP_API_RANGE("sp_mttkrp");
     if (!T || !B || !C || !M || R < 1) return SP_ERR_INVALID_ARG;
     if (T->rank != 3 || T->ord[0] != 0 || T->lt[1] != SP_COMPRESSED || T->lt[2] != SP_COMPRESSED)
         return SP_ERR_UNSUPPORTED;
@@ -398,6 +399,7 @@ extern "C" sp_status sp_mttkrp(sp_tensor* T, const double* B, const double* C, i
 
 extern "C" sp_status sp_mttkrp_mode(sp_tensor* T, int mode, const double* const* factors, int64_t R, double* M,
                                     void* stream_) {
+    SP_API_RANGE("sp_mttkrp_mode");
     if (!T || !factors || !M || R < 1 || mode < 0 || mode > 2) return SP_ERR_INVALID_ARG;
     if (T->rank != 3 || T->ord[0] != mode || T->lt[1] != SP_COMPRESSED || T->lt[2] != SP_COMPRESSED)
         return SP_ERR_UNSUPPORTED;
@@ -408,6 +410,7 @@ extern "C" sp_status sp_mttkrp_mode(sp_tensor* T, int mode, const double* const*
 }
 
 static sp_status mttkrp_levels(sp_tensor* T, const double* F1, const double* F2, int64_t R, double* M, cudaStream_t stream) {
+    if (sp_check_device(T) != SP_OK) return SP_ERR_INVALID_ARG;
     {   // 8- and 16-bit storage is read through its 32-bit shadow
         sp_tensor* wide_ = nullptr;
         const sp_status ws_ = sp_widened(T, stream, &wide_);

@@ -24,18 +24,22 @@ namespace {
 constexpr int kErrRange = 1;
 constexpr int kErrDup = 2;
 
-// Optional phase timing of sp_pack (sp_set_profiling): CUDA events on the caller's stream.
+// Phase timing of the packer: CUDA events on the caller's stream between its kernels.  The product
+// library never asks for it (times == nullptr: no event is created); the benchmark's own library
+// compiles this file a second time with SP_BENCH_BUILD and exports the timed variant.
 enum { kPhKeys = 0, kPhUpsweep, kPhScan, kPhDownsweep, kPhCount, kPhEmit, kPhCount_ };
-bool g_profiling = false;
-double g_phase_ms[SP_PACK_PROFILE_LEN] = {0, 0, 0, 0, 0, 0};
-int g_phase_passes = 0;
+struct PackTimes {
+    double ms[kPhCount_];
+    int passes;
+};
 
 struct PhaseTimer {
     cudaStream_t stream;
+    PackTimes* out;
     bool on;
     std::vector<cudaEvent_t> ev;
     std::vector<int> phase;
-    PhaseTimer(cudaStream_t s, bool enabled) : stream(s), on(enabled) { if (on) mark(-1); }
+    PhaseTimer(cudaStream_t s, PackTimes* times) : stream(s), out(times), on(times != nullptr) { if (on) mark(-1); }
     // closes the interval that started at the previous mark and files it under `ph`
     void mark(int ph) {
         if (!on) return;
@@ -48,13 +52,13 @@ struct PhaseTimer {
     void finish(int passes) {
         if (!on) return;
         cudaEventSynchronize(ev.back());
-        for (int i = 0; i < SP_PACK_PROFILE_LEN; ++i) g_phase_ms[i] = 0;
+        for (int i = 0; i < kPhCount_; ++i) out->ms[i] = 0;
         for (size_t i = 1; i < ev.size(); ++i) {
             float ms = 0;
             cudaEventElapsedTime(&ms, ev[i - 1], ev[i]);
-            if (phase[i] >= 0) g_phase_ms[phase[i]] += ms;
+            if (phase[i] >= 0) out->ms[phase[i]] += ms;
         }
-        g_phase_passes = passes;
+        out->passes = passes;
     }
     ~PhaseTimer() { for (auto e : ev) cudaEventDestroy(e); }
 };
@@ -631,13 +635,11 @@ int ceil_log2(int64_t v) {   // bits needed for coordinates 0..v-1
     return b;
 }
 
-}  // namespace
-
 // ---------------------------------------------------------------------------
-extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const void* const* coo_coords,
-                             int coo_coord_bits, const double* coo_vals, const sp_level_type* dimLevelType,
-                             const int* dimOrdering, int posBits, int crdBits, unsigned flags, void* stream_,
-                             sp_tensor** out) {
+sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* const* coo_coords,
+                    int coo_coord_bits, const double* coo_vals, const sp_level_type* dimLevelType,
+                    const int* dimOrdering, int posBits, int crdBits, unsigned flags, void* stream_,
+                    sp_tensor** out, PackTimes* times) {
     if (!out) return SP_ERR_INVALID_ARG;
     *out = nullptr;
     if (rank < 1 || rank > SP_MAX_RANK || !dims || !dimLevelType || nnz < 0) return SP_ERR_INVALID_ARG;
@@ -677,7 +679,7 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
         if (plan.lt[l] == SP_COMPRESSED && (uint64_t)(plan.sz[l] - 1) > max_crd) return SP_ERR_WIDTH_OVERFLOW;
 
     sp_workspace ws(stream);
-    PhaseTimer timer(stream, g_profiling);
+    PhaseTimer timer(stream, times);
     int npasses_done = 0;
     const int64_t n = nnz;
     int64_t counts[SP_MAX_RANK] = {};
@@ -845,20 +847,37 @@ extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const v
     return SP_OK;
 }
 
-extern "C" sp_status sp_set_profiling(int enabled) {
-    g_profiling = enabled != 0;
-    return SP_OK;
-}
+}  // namespace
 
-extern "C" sp_status sp_get_pack_profile(double* ms, int* npasses) {
-    if (!ms) return SP_ERR_INVALID_ARG;
-    for (int i = 0; i < SP_PACK_PROFILE_LEN; ++i) ms[i] = g_phase_ms[i];
-    if (npasses) *npasses = g_phase_passes;
-    return SP_OK;
+#ifdef SP_BENCH_BUILD
+// The benchmark's library: the same packer with its phases bracketed by events.
+// phase_ms: host, 6 entries (key build, sort histograms, sort scans, sort scatters, node counting,
+// emit + fill); npasses: host, number of radix passes.
+extern "C" sp_status spb_pack_timed(int rank, const int64_t* dims, int64_t nnz, const void* const* coo_coords,
+                                    int coo_coord_bits, const double* coo_vals, const sp_level_type* dimLevelType,
+                                    const int* dimOrdering, int posBits, int crdBits, unsigned flags, void* stream_,
+                                    sp_tensor** out, double* phase_ms, int* npasses) {
+    if (!phase_ms) return SP_ERR_INVALID_ARG;
+    PackTimes t = {};
+    const sp_status st = pack_impl(rank, dims, nnz, coo_coords, coo_coord_bits, coo_vals, dimLevelType, dimOrdering,
+                                   posBits, crdBits, flags, stream_, out, &t);
+    for (int i = 0; i < kPhCount_; ++i) phase_ms[i] = t.ms[i];
+    if (npasses) *npasses = t.passes;
+    return st;
+}
+#else
+extern "C" sp_status sp_pack(int rank, const int64_t* dims, int64_t nnz, const void* const* coo_coords,
+                             int coo_coord_bits, const double* coo_vals, const sp_level_type* dimLevelType,
+                             const int* dimOrdering, int posBits, int crdBits, unsigned flags, void* stream_,
+                             sp_tensor** out) {
+    SP_API_RANGE("sp_pack");
+    return pack_impl(rank, dims, nnz, coo_coords, coo_coord_bits, coo_vals, dimLevelType, dimOrdering, posBits,
+                     crdBits, flags, stream_, out, nullptr);
 }
 
 extern "C" sp_status sp_unpack(const sp_tensor* t, void* const* coo_coords_out, double* vals_out,
                                int64_t* nnz_out, void* stream_) {
+    SP_API_RANGE("sp_unpack");
     if (!t || !coo_coords_out || !vals_out || !nnz_out) return SP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     UnpackArgs a;
@@ -892,6 +911,7 @@ extern "C" sp_status sp_unpack(const sp_tensor* t, void* const* coo_coords_out, 
 // through an intermediate coordinate scheme rather than one direct converter per pair of formats).
 extern "C" sp_status sp_convert(const sp_tensor* t, const sp_level_type* dimLevelType, const int* dimOrdering,
                                 int posBits, int crdBits, void* stream_, sp_tensor** out) {
+    SP_API_RANGE("sp_convert");
     if (!out) return SP_ERR_INVALID_ARG;
     *out = nullptr;
     if (!t || !dimLevelType) return SP_ERR_INVALID_ARG;
@@ -908,3 +928,4 @@ extern "C" sp_status sp_convert(const sp_tensor* t, const sp_level_type* dimLeve
     return sp_pack(t->rank, t->dims, cnt, coords, 64, vals, dimLevelType, dimOrdering, posBits, crdBits, SP_DUP_SUM,
                    stream_, out);
 }
+#endif  // SP_BENCH_BUILD

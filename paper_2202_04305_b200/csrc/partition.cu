@@ -67,7 +67,10 @@ sp_status sp_get_segment_ids(sp_tensor* t, cudaStream_t stream, const uint32_t**
     std::lock_guard<std::mutex> lock(t->mu);
     const uint64_t key = (uint64_t)SP_PART_SEGIDS << 56;
     auto it = t->parts.find(key);
-    if (it != t->parts.end()) { *out = reinterpret_cast<const uint32_t*>(it->second.aux); return SP_OK; }
+    if (it != t->parts.end()) {
+        *out = reinterpret_cast<const uint32_t*>(it->second.aux);
+        return sp_partition_wait(it->second, stream);
+    }
     const int64_t nseg = t->npos[1] - 1, nnz = t->ncrd[1];
     sp_partition p;
     p.aux = static_cast<int64_t*>(sp_dev_alloc((size_t)(nnz ? nnz : 1) * sizeof(uint32_t), stream));
@@ -80,20 +83,20 @@ sp_status sp_get_segment_ids(sp_tensor* t, cudaStream_t stream, const uint32_t**
                                                            t->lt[0] == SP_COMPRESSED ? static_cast<const I*>(t->crd[0]) : nullptr,
                                                            seg);
         });
-        SP_LAUNCH_CHECK();
+        if (cudaGetLastError() != cudaSuccess) { sp_dev_free(p.aux, stream); return SP_ERR_CUDA; }
         sp_count_launches(1);
     }
+    if (sp_partition_built(&p, stream) != SP_OK) { sp_dev_free(p.aux, stream); return SP_ERR_CUDA; }
     t->parts[key] = p;
     *out = seg;
     return SP_OK;
 }
 
-sp_status sp_get_merge_partition(sp_tensor* t, int64_t items, int64_t carry_elems_per_chunk, cudaStream_t stream,
-                                 sp_partition* out) {
+sp_status sp_get_merge_partition(sp_tensor* t, int64_t items, cudaStream_t stream, sp_partition* out) {
     std::lock_guard<std::mutex> lock(t->mu);
-    const uint64_t key = ((uint64_t)SP_PART_MERGE_LAST << 56) | ((uint64_t)carry_elems_per_chunk << 32) | (uint64_t)items;
+    const uint64_t key = ((uint64_t)SP_PART_MERGE_LAST << 56) | (uint64_t)items;
     auto it = t->parts.find(key);
-    if (it != t->parts.end()) { *out = it->second; return SP_OK; }
+    if (it != t->parts.end()) { *out = it->second; return sp_partition_wait(it->second, stream); }
     const int last = t->rank - 1;
     const int64_t nseg = t->npos[last] - 1;
     const int64_t nnz = t->ncrd[last];
@@ -102,13 +105,8 @@ sp_status sp_get_merge_partition(sp_tensor* t, int64_t items, int64_t carry_elem
     if (p.nchunks < 1) p.nchunks = 1;
     p.row = static_cast<int64_t*>(sp_dev_alloc((size_t)(p.nchunks + 1) * sizeof(int64_t), stream));
     p.nz = static_cast<int64_t*>(sp_dev_alloc((size_t)(p.nchunks + 1) * sizeof(int64_t), stream));
-    p.carry_elems = p.nchunks * (carry_elems_per_chunk + 1);
-    // carry: per chunk `carry_elems_per_chunk` doubles, then one int64 row id per chunk
-    p.carry = static_cast<double*>(sp_dev_alloc((size_t)p.carry_elems * sizeof(double), stream));
-    if (!p.row || !p.nz || !p.carry) {
-        sp_dev_free(p.row, stream); sp_dev_free(p.nz, stream); sp_dev_free(p.carry, stream);
-        return SP_ERR_ALLOC;
-    }
+    auto drop = [&](sp_status s) { sp_dev_free(p.row, stream); sp_dev_free(p.nz, stream); return s; };
+    if (!p.row || !p.nz) return drop(SP_ERR_ALLOC);
     const unsigned blocks = (unsigned)sp_ceil_div(p.nchunks + 1, 256);
     if (t->posBits == 32)
         k_merge_partition<uint32_t><<<blocks, 256, 0, stream>>>(static_cast<const uint32_t*>(t->pos[last]), nseg, nnz,
@@ -116,8 +114,9 @@ sp_status sp_get_merge_partition(sp_tensor* t, int64_t items, int64_t carry_elem
     else
         k_merge_partition<uint64_t><<<blocks, 256, 0, stream>>>(static_cast<const uint64_t*>(t->pos[last]), nseg, nnz,
                                                                  items, p.nchunks, p.row, p.nz);
-    SP_LAUNCH_CHECK();
+    if (cudaGetLastError() != cudaSuccess) return drop(SP_ERR_CUDA);
     sp_count_launches(1);
+    if (sp_partition_built(&p, stream) != SP_OK) return drop(SP_ERR_CUDA);
     t->parts[key] = p;
     *out = p;
     return SP_OK;
@@ -156,7 +155,11 @@ sp_status widen_array(const void* src, int64_t n, int bits, cudaStream_t stream,
 sp_status sp_widened(sp_tensor* t, cudaStream_t stream, sp_tensor** out) {
     if (t->posBits >= 32 && t->crdBits >= 32) { *out = t; return SP_OK; }
     std::lock_guard<std::mutex> lock(t->mu);
-    if (t->wide) { *out = t->wide; return SP_OK; }
+    if (t->wide) {
+        *out = t->wide;
+        if (t->wide_ready && stream != t->wide_built_on) SP_CUDA(cudaStreamWaitEvent(stream, t->wide_ready, 0));
+        return SP_OK;
+    }
     sp_tensor* w = new sp_tensor();
     w->rank = t->rank;
     w->device = t->device;
@@ -173,6 +176,9 @@ sp_status sp_widened(sp_tensor* t, cudaStream_t stream, sp_tensor** out) {
         if (st == SP_OK) st = widen_array(t->crd[l], t->ncrd[l], t->crdBits, stream, &w->crd[l]);
     }
     if (st != SP_OK) { sp_free(w); return st; }
+    if (cudaEventCreateWithFlags(&t->wide_ready, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventRecord(t->wide_ready, stream) != cudaSuccess) { sp_free(w); return SP_ERR_CUDA; }
+    t->wide_built_on = stream;
     t->wide = w;
     *out = w;
     return SP_OK;
@@ -182,7 +188,7 @@ sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t per, cudaStream_t stream
     std::lock_guard<std::mutex> lock(t->mu);
     const uint64_t key = ((uint64_t)SP_PART_MTTKRP << 56) | (uint64_t)per;
     auto it = t->parts.find(key);
-    if (it != t->parts.end()) { *out = it->second; return SP_OK; }
+    if (it != t->parts.end()) { *out = it->second; return sp_partition_wait(it->second, stream); }
     const int64_t nnz = t->ncrd[2];
     const int64_t nfiber = t->ncrd[1];
     const int64_t nslice = t->npos[1] - 1;
@@ -192,10 +198,8 @@ sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t per, cudaStream_t stream
     p.row = static_cast<int64_t*>(sp_dev_alloc((size_t)(p.nchunks + 1) * sizeof(int64_t), stream));
     p.nz = static_cast<int64_t*>(sp_dev_alloc((size_t)(p.nchunks + 1) * sizeof(int64_t), stream));
     p.aux = static_cast<int64_t*>(sp_dev_alloc((size_t)(p.nchunks + 1) * sizeof(int64_t), stream));
-    if (!p.row || !p.nz || !p.aux) {
-        sp_dev_free(p.row, stream); sp_dev_free(p.nz, stream); sp_dev_free(p.aux, stream);
-        return SP_ERR_ALLOC;
-    }
+    auto drop = [&](sp_status s) { sp_dev_free(p.row, stream); sp_dev_free(p.nz, stream); sp_dev_free(p.aux, stream); return s; };
+    if (!p.row || !p.nz || !p.aux) return drop(SP_ERR_ALLOC);
     const unsigned blocks = (unsigned)sp_ceil_div(p.nchunks + 1, 256);
     if (t->posBits == 32)
         k_mttkrp_partition<uint32_t><<<blocks, 256, 0, stream>>>(
@@ -205,8 +209,9 @@ sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t per, cudaStream_t stream
         k_mttkrp_partition<uint64_t><<<blocks, 256, 0, stream>>>(
             static_cast<const uint64_t*>(t->pos[1]), nslice, static_cast<const uint64_t*>(t->pos[2]), nfiber, nnz, per,
             p.nchunks, p.row, p.nz, p.aux);
-    SP_LAUNCH_CHECK();
+    if (cudaGetLastError() != cudaSuccess) return drop(SP_ERR_CUDA);
     sp_count_launches(1);
+    if (sp_partition_built(&p, stream) != SP_OK) return drop(SP_ERR_CUDA);
     t->parts[key] = p;
     *out = p;
     return SP_OK;

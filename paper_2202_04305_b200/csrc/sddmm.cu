@@ -206,7 +206,9 @@ sp_status sddmm_dense_inner(sp_tensor* S, const double* A, int64_t lda, const do
 
 extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const double* B, int64_t ldb, int64_t K,
                               double* x_vals, void* stream_) {
+    SP_API_RANGE("sp_sddmm");
     if (!S || !A || !B || K < 1 || lda < K) return SP_ERR_INVALID_ARG;
+    if (sp_check_device(S) != SP_OK) return SP_ERR_INVALID_ARG;
     {   // 8- and 16-bit storage is read through its 32-bit shadow
         sp_tensor* wide_ = nullptr;
         const sp_status ws_ = sp_widened(S, static_cast<cudaStream_t>(stream_), &wide_);
@@ -235,7 +237,7 @@ extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const 
     SP_LAUNCH_CHECK();
 
     sp_partition part;
-    sp_status st = sp_get_merge_partition(S, kSItems, 0, stream, &part);
+    sp_status st = sp_get_merge_partition(S, kSItems, stream, &part);
     if (st != SP_OK) return st;
     const bool vec2 = (K % 2 == 0) && (lda % 2 == 0) && (reinterpret_cast<uintptr_t>(A) % 16 == 0) &&
                       (reinterpret_cast<uintptr_t>(Bt) % 16 == 0);

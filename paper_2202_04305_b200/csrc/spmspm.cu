@@ -157,6 +157,7 @@ k_row_offsets(const int64_t* __restrict__ rowlen, int64_t m, void* __restrict__ 
 
 extern "C" sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBits, int crdBits, void* stream_,
                                sp_tensor** out) {
+    SP_API_RANGE("sp_spmspm");
     if (!out) return SP_ERR_INVALID_ARG;
     *out = nullptr;
     if (!A || !B) return SP_ERR_INVALID_ARG;

@@ -199,93 +199,6 @@ __device__ __forceinline__ void st_vec(double* p, const double* a) {
     else *p = a[0];
 }
 
-template <typename P, typename I, int V, bool SCATTER>
-__global__ void __launch_bounds__(kMThreads)
-k_spmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
-       const I* __restrict__ outer, const double* __restrict__ B, int64_t N, int64_t ldb,
-       double* __restrict__ C, int64_t ldc, const int64_t* __restrict__ prow, const int64_t* __restrict__ pnz,
-       int64_t nchunks, int64_t nseg, double* __restrict__ carry, int64_t* __restrict__ carry_row) {
-    const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
-    if (w >= nchunks) return;
-    const int lane = threadIdx.x & 31;
-    const int64_t i0 = prow[w], j0 = pnz[w], i1 = prow[w + 1], j1 = pnz[w + 1];
-    int64_t pstart = j0;
-
-    for (int64_t cbase = 0; cbase < N; cbase += 32 * V) {
-        const int64_t col = cbase + (int64_t)lane * V;
-        const bool on = col < N;
-        double acc[V];
-#pragma unroll
-        for (int q = 0; q < V; ++q) acc[q] = 0.0;
-        int64_t row = i0, p = j0, rbase = i0, nzbase = j0;
-        pstart = j0;
-        int64_t E = (rbase + lane < i1) ? (int64_t)pos[rbase + lane + 1] : j1;
-        I c_l = (nzbase + lane < j1) ? crd[nzbase + lane] : (I)0;
-        double v_l = (nzbase + lane < j1) ? val[nzbase + lane] : 0.0;
-        vec_t<V> brow;
-#pragma unroll
-        for (int q = 0; q < V; ++q) brow.a[q] = 0.0;
-        if (SCATTER && on && row < nseg) brow = ld_vec<V>(B + (outer ? (int64_t)outer[row] : row) * ldb + col);
-
-        while (true) {
-            const int64_t rend = row < i1 ? __shfl_sync(0xffffffffu, E, (int)(row - rbase)) : j1;
-            while (p < rend) {
-                int off = (int)(p - nzbase);
-                if (off == 32) {
-                    nzbase += 32;
-                    c_l = (nzbase + lane < j1) ? crd[nzbase + lane] : (I)0;
-                    v_l = (nzbase + lane < j1) ? val[nzbase + lane] : 0.0;
-                    off = 0;
-                }
-                const int cnt = (int)min(rend - p, (int64_t)(32 - off));
-                for (int t = 0; t < cnt; t += 4) {
-                    vec_t<V> b[4];
-                    double vv[4];
-                    int64_t kk[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        vv[u] = 0.0;
-                        kk[u] = 0;
-#pragma unroll
-                        for (int q = 0; q < V; ++q) b[u].a[q] = 0.0;
-                        if (t + u < cnt) {
-                            kk[u] = (int64_t)__shfl_sync(0xffffffffu, c_l, off + t + u);
-                            vv[u] = __shfl_sync(0xffffffffu, v_l, off + t + u);
-                            if (!SCATTER && on) b[u] = ld_vec<V>(B + kk[u] * ldb + col);
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        if (SCATTER) {
-                            if (t + u < cnt && on) {
-#pragma unroll
-                                for (int q = 0; q < V; ++q) atomicAdd(C + kk[u] * ldc + col + q, vv[u] * brow.a[q]);
-                            }
-                        } else {
-#pragma unroll
-                            for (int q = 0; q < V; ++q) acc[q] = fma(vv[u], b[u].a[q], acc[q]);
-                        }
-                    }
-                }
-                p += cnt;
-            }
-            if (row >= i1) break;
-            if (!SCATTER && on) st_vec<V>(C + (outer ? (int64_t)outer[row] : row) * ldc + col, acc);
-#pragma unroll
-            for (int q = 0; q < V; ++q) acc[q] = 0.0;
-            ++row;
-            pstart = p;
-            if (row - rbase == 32) {
-                rbase += 32;
-                E = (rbase + lane < i1) ? (int64_t)pos[rbase + lane + 1] : j1;
-            }
-            if (SCATTER && on && row < nseg) brow = ld_vec<V>(B + (outer ? (int64_t)outer[row] : row) * ldb + col);
-        }
-        if (!SCATTER && on && j1 > pstart) st_vec<V>(carry + w * N + col, acc);
-    }
-    if (!SCATTER && lane == 0) carry_row[w] = (j1 > pstart && i1 < nseg) ? i1 : -1;
-}
-
 // Row-major SpMM (CSR, DCSR).  A warp walks its merge-path piece 32 entries at a time; lane = output
 // column(s).  The ends of the rows that fall inside a batch come from a 32-row window of pos[] as a
 // bit mask, so the loads of the batch do not depend on the row structure: B rows are fetched in
@@ -466,7 +379,9 @@ bool matrix_encoding_ok(const sp_tensor* A) {
 }  // namespace
 
 extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* stream_) {
+    SP_API_RANGE("sp_spmv");
     if (!A || !x || !y) return SP_ERR_INVALID_ARG;
+    if (sp_check_device(A) != SP_OK) return SP_ERR_INVALID_ARG;
     {   // 8- and 16-bit storage is read through its 32-bit shadow
         sp_tensor* wide_ = nullptr;
         const sp_status ws_ = sp_widened(A, static_cast<cudaStream_t>(stream_), &wide_);
@@ -484,10 +399,13 @@ extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* str
     const int64_t nseg = A->npos[1] - 1;
     if (nseg <= 0) return SP_OK;
     sp_partition part;
-    sp_status st = sp_get_merge_partition(A, kVTile, 1, stream, &part);
+    sp_status st = sp_get_merge_partition(A, kVTile, stream, &part);
     if (st != SP_OK) return st;
-    double* cval = part.carry;
-    int64_t* crow = reinterpret_cast<int64_t*>(part.carry + part.nchunks);
+    // the open row of every tile: its partial sum and its row number, scratch of this call alone
+    sp_workspace ws(stream);
+    double* cval = rowmajor ? ws.get<double>((size_t)part.nchunks) : nullptr;
+    int64_t* crow = rowmajor ? ws.get<int64_t>((size_t)part.nchunks) : nullptr;
+    if (ws.failed) return SP_ERR_ALLOC;
     SP_DISPATCH_WIDTHS(A, {
         const P* pos = static_cast<const P*>(A->pos[1]);
         const I* crd = static_cast<const I*>(A->crd[1]);
@@ -509,7 +427,9 @@ extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* str
 
 extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t ldb, double* C, int64_t ldc,
                              void* stream_) {
+    SP_API_RANGE("sp_spmm");
     if (!A || !B || !C || N < 1 || ldb < N || ldc < N) return SP_ERR_INVALID_ARG;
+    if (sp_check_device(A) != SP_OK) return SP_ERR_INVALID_ARG;
     if (N >= (1 << 20)) return SP_ERR_UNSUPPORTED;
     {   // 8- and 16-bit storage is read through its 32-bit shadow
         sp_tensor* wide_ = nullptr;
@@ -531,26 +451,29 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
     const int64_t nseg = A->npos[1] - 1;
     if (nseg <= 0) return SP_OK;
     // column-major storage runs as a flat loop over entries with their column ids expanded once
+    // (32-bit ids: a column-major matrix with 2^32 or more columns is refused)
+    if (!rowmajor && A->dims[1] >= ((int64_t)1 << 32)) return SP_ERR_UNSUPPORTED;
     const uint32_t* segs = nullptr;
     sp_status st = SP_OK;
-    if (!rowmajor && A->dims[1] < ((int64_t)1 << 32)) {
+    sp_partition part;
+    sp_workspace ws(stream);
+    double* carry = nullptr;
+    int64_t* crow = nullptr;
+    if (!rowmajor) {
         st = sp_get_segment_ids(A, stream, &segs);
         if (st != SP_OK) return st;
-    }
-    sp_partition part;
-    if (!segs) {
-        st = sp_get_merge_partition(A, kMItems, N, stream, &part);
+    } else {
+        st = sp_get_merge_partition(A, kMItems, stream, &part);
         if (st != SP_OK) return st;
+        // the open row of every warp's piece: N partial sums and the row number, scratch of this call alone
+        carry = ws.get<double>((size_t)part.nchunks * N);
+        crow = ws.get<int64_t>((size_t)part.nchunks);
+        if (ws.failed) return SP_ERR_ALLOC;
     }
-    double* carry = part.carry;
-    int64_t* crow = reinterpret_cast<int64_t*>(part.carry + part.nchunks * N);
     const bool vec2 = N > 32 && (N % 2 == 0) && (ldb % 2 == 0) && (ldc % 2 == 0) &&
                       (reinterpret_cast<uintptr_t>(B) % 16 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0) &&
                       (reinterpret_cast<uintptr_t>(carry) % 16 == 0);
     const unsigned blocks = (unsigned)sp_ceil_div(part.nchunks * 32, kMThreads);
-#define SP_SPMM_LAUNCH(V, SC)                                                                                   \
-    k_spmm<P, I, V, SC><<<blocks, kMThreads, 0, stream>>>(pos, crd, A->val, outer, B, N, ldb, C, ldc, part.row, \
-                                                          part.nz, part.nchunks, nseg, carry, crow)
     SP_DISPATCH_WIDTHS(A, {
         const P* pos = static_cast<const P*>(A->pos[1]);
         const I* crd = static_cast<const I*>(A->crd[1]);
@@ -564,7 +487,8 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
                                                                          part.nz, part.nchunks, nseg, carry, crow);
             k_spmm_fixup<I><<<blocks, kMThreads, 0, stream>>>(carry, crow, part.nchunks, outer, N, C, ldc);
             sp_count_launches(2);
-        } else if (segs) {
+        } else {
+            (void)pos;
             const int64_t nnz = A->ncrd[1];
             const unsigned sblocks = (unsigned)sp_ceil_div(sp_ceil_div(nnz, kScatPer) * 32, kMThreads);
             if (nnz > 0) {
@@ -572,12 +496,8 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
                 else k_spmm_scatter<I, 1><<<sblocks, kMThreads, 0, stream>>>(segs, crd, A->val, nnz, B, N, ldb, C, ldc);
                 sp_count_launches(1);
             }
-        } else {
-            if (vec2) SP_SPMM_LAUNCH(2, true); else SP_SPMM_LAUNCH(1, true);
-            sp_count_launches(1);
         }
     });
-#undef SP_SPMM_LAUNCH
     SP_LAUNCH_CHECK();
     return SP_OK;
 }
@@ -640,7 +560,9 @@ __global__ void k_static_partition(const P* __restrict__ pos, int64_t nseg, int6
 }  // namespace
 
 extern "C" sp_status sp_spmv_static(const sp_tensor* A, const double* x, double* y, void* stream_) {
+    SP_API_RANGE("sp_spmv_static");
     if (!A || !x || !y) return SP_ERR_INVALID_ARG;
+    if (sp_check_device(A) != SP_OK) return SP_ERR_INVALID_ARG;
     if (!matrix_encoding_ok(A)) return SP_ERR_UNSUPPORTED;
     if (A->posBits < 32 || A->crdBits < 32) return SP_ERR_UNSUPPORTED;   // a widened copy would need an allocation
     const int64_t nseg = A->npos[1] - 1;

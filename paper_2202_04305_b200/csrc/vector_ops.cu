@@ -43,6 +43,7 @@ k_vec_dot(const I* __restrict__ acrd, const double* __restrict__ aval, int64_t n
 }  // namespace
 
 extern "C" sp_status sp_scale(sp_tensor* x, double c, void* stream_) {
+    SP_API_RANGE("sp_scale");
     if (!x) return SP_ERR_INVALID_ARG;
     if (x->nval > 0) {
         k_scale<<<(unsigned)sp_ceil_div(x->nval, 256), 256, 0, static_cast<cudaStream_t>(stream_)>>>(x->val, x->nval, c);
@@ -53,6 +54,7 @@ extern "C" sp_status sp_scale(sp_tensor* x, double c, void* stream_) {
 }
 
 extern "C" sp_status sp_vec_dot(const sp_tensor* a, const sp_tensor* b, double* result, void* stream_) {
+    SP_API_RANGE("sp_vec_dot");
     if (!a || !b || !result) return SP_ERR_INVALID_ARG;
     if (a->rank != 1 || b->rank != 1 || a->lt[0] != SP_COMPRESSED || b->lt[0] != SP_COMPRESSED) return SP_ERR_UNSUPPORTED;
     if (a->crdBits != b->crdBits) return SP_ERR_UNSUPPORTED;

@@ -192,3 +192,32 @@ def test_sparse_dot_by_co_iteration(oracle, n, na, nb):
     assert abs(x - float(da @ db)) <= 1e-12 * float(np.abs(da) @ np.abs(db)) + 0.0
     assert np.isclose(bd, float(np.abs(da) @ np.abs(db)), rtol=1e-13, atol=0)
     assert oracle.vec_dot(a.coords[0][oa], a.vals[oa], a.coords[0][oa], np.ones(na))[0] == pytest.approx(a.vals.sum(), abs=1e-12)
+
+
+@pytest.mark.parametrize("lt", [(0, 1), (1, 1)])
+def test_storage_loop_nests_match_the_coordinate_loops(oracle, lt):
+    """The all-cores baseline loops (over packed storage) against the coordinate-loop definitions."""
+    coo = I.confined_rows_matrix(60, 40, 300, row_fraction=0.5, seed=21)
+    s = oracle.pack(coo.dims, coo.coords, coo.vals, lt)
+    B = I.dense_operand(3, 61, 40, 7)
+    ref, bd = oracle.spmm(60, coo.coords[0], coo.coords[1], coo.vals, B)
+    got, nt = oracle.par_spmm(s, B)
+    assert nt >= 1 and np.all(np.abs(got - ref) <= 1e-15 * bd) and np.all(got[bd == 0] == 0)
+    x = I.uniform_pm1(3, 62, 40)
+    yref, yb = oracle.spmv(60, coo.coords[0], coo.coords[1], coo.vals, x)
+    assert np.all(np.abs(oracle.par_spmv(s, x)[0] - yref) <= 1e-15 * yb)
+    A = I.dense_operand(3, 63, 60, 9)
+    Bk = I.dense_operand(3, 64, 9, 40)
+    xe, xb = oracle.sddmm(coo.coords[0], coo.coords[1], coo.vals, A, Bk)
+    xs, _ = oracle.par_sddmm(s, A, Bk)
+    assert np.all(np.abs(xs[s.entry_pos] - xe) <= 1e-15 * xb)
+
+
+@pytest.mark.parametrize("lt", [(0, 1, 1), (1, 1, 1)])
+def test_storage_mttkrp_matches_the_coordinate_loop(oracle, lt):
+    t = I.zipf_tensor3(12, 400, seed=22)
+    s = oracle.pack(t.dims, t.coords, t.vals, lt)
+    Bf, Cf = I.dense_operand(3, 65, 12, 6), I.dense_operand(3, 66, 12, 6)
+    ref, bd = oracle.mttkrp(12, *t.coords, t.vals, Bf, Cf)
+    got, nt = oracle.par_mttkrp(s, Bf, Cf)
+    assert nt >= 1 and np.all(np.abs(got - ref) <= 1e-15 * bd) and np.all(got[bd == 0] == 0)

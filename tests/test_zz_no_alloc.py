@@ -24,14 +24,17 @@ def _both(A, x):
     return y.cpu().numpy(), y_ref.cpu().numpy()
 
 
+@pytest.mark.parametrize("widths", [(32, 32), (64, 64), (32, 64), (64, 32)])
 @pytest.mark.parametrize("enc", list(MATRIX_ENCODINGS))
-def test_static_matches_spmv_two_calls_in_a_row(oracle, enc):
+def test_static_matches_spmv_two_calls_in_a_row(oracle, enc, widths):
     lt, od = MATRIX_ENCODINGS[enc]
+    if widths != (32, 32) and enc in ("DCSR", "CSC"):
+        pytest.skip("the mixed and wide width pairs run on the CSR and DCSC encodings")
     big = I.config2(seed=11, n=6000)                       # about 47 tiles, power-law rows
     small = I.row_band_matrix(900, 7, seed=12)             # rows longer than a tile's share, many empty rows
     for coo, xs in ((big, 41), (small, 42)):               # two calls back to back per matrix, four in all
         coords, vals = to_dev(coo)
-        A = sp().sp_pack(coo.dims, coords, vals, lt, od)
+        A = sp().sp_pack(coo.dims, coords, vals, lt, od, posBits=widths[0], crdBits=widths[1])
         for rep in range(2):
             x = I.uniform_pm1(13, xs + 10 * rep, coo.dims[1])
             got, ref = _both(A, dev(x))
