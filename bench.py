@@ -53,7 +53,7 @@ def build_probes(force: bool = False) -> str:
         return PROBE_LIB
     cmd = [libbuild._nvcc(), "-Wno-deprecated-gpu-targets", "-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-Xcompiler", "-fPIC", "-diag-suppress", "177", "-DSP_BENCH_BUILD", "-I", os.path.join(ROOT, "include"), "-I", ROOT,
-           "-I", os.path.join(pkg, "csrc"), "-shared", "-o", PROBE_LIB] + srcs + \
+           "-I", os.path.join(pkg, "csrc"), "-shared", "-o", PROBE_LIB] + os.environ.get("SP_NVCC_FLAGS", "").split() + srcs + \
           ["-L" + pkg, "-lsp", "-Xlinker", "-rpath=$ORIGIN/" + os.path.basename(pkg), "-lcudart"]
     subprocess.check_call(cmd)
     return PROBE_LIB

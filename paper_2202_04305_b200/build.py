@@ -14,6 +14,8 @@ LIB = os.path.join(HERE, "libsp.so")
 SOURCES = ["api.cu", "pack.cu", "partition.cu", "spmv_spmm.cu", "sddmm.cu", "mttkrp.cu", "dense_inner.cu", "spmspm.cu", "vector_ops.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+# extra compiler flags, e.g. SP_NVCC_FLAGS="-DSP_SORT_MAX_BITS=8"; a change of them needs --force
+NVCC_FLAGS += os.environ.get("SP_NVCC_FLAGS", "").split()
 
 
 def _nvcc() -> str:

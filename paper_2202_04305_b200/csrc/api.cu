@@ -41,9 +41,22 @@ sp_status sp_partition_built(sp_partition* p, cudaStream_t stream) {
     return SP_OK;
 }
 
-sp_status sp_partition_wait(const sp_partition& p, cudaStream_t stream) {
-    if (p.ready && stream != p.built_on) SP_CUDA(cudaStreamWaitEvent(stream, p.ready, 0));
+sp_status sp_event_wait(cudaEvent_t ready, cudaStream_t built_on, cudaStream_t stream) {
+    if (!ready || stream == built_on) return SP_OK;
+    const cudaError_t q = cudaEventQuery(ready);
+    if (q == cudaSuccess) return SP_OK;                 // the table was finished long ago: nothing to wait for
+    if (q != cudaErrorNotReady) { cudaGetLastError(); return SP_ERR_CUDA; }
+    cudaGetLastError();
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    SP_CUDA(cudaStreamIsCapturing(stream, &cap));
+    // a stream that is being captured cannot wait for work outside its graph: finish that work first
+    if (cap != cudaStreamCaptureStatusNone) SP_CUDA(cudaEventSynchronize(ready));
+    else SP_CUDA(cudaStreamWaitEvent(stream, ready, 0));
     return SP_OK;
+}
+
+sp_status sp_partition_wait(const sp_partition& p, cudaStream_t stream) {
+    return sp_event_wait(p.ready, p.built_on, stream);
 }
 
 extern "C" {

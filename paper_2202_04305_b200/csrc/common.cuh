@@ -47,6 +47,7 @@ struct sp_tensor {
     // For handles stored with 8- or 16-bit positions/coordinates: a copy of the overhead arrays
     // widened to 32 bits that the compute kernels read (values shared, not copied).  Built on
     // first use by sp_widened(), owned by this handle.
+    int64_t max_seg = -1;      // longest segment of the last level (entries under one parent); -1 = not measured yet
     sp_tensor* wide = nullptr;
     cudaEvent_t wide_ready = nullptr;
     cudaStream_t wide_built_on = nullptr;
@@ -57,8 +58,9 @@ struct sp_tensor {
 sp_status sp_check_device(const sp_tensor* t);
 // Marks the end of the work that fills a cached table (p->ready, p->built_on).
 sp_status sp_partition_built(sp_partition* p, cudaStream_t stream);
-// Makes `stream` wait for that work when it is not the stream that did it.
+// Makes `stream` wait for that work when it is not the stream that did it (and it is still running).
 sp_status sp_partition_wait(const sp_partition& p, cudaStream_t stream);
+sp_status sp_event_wait(cudaEvent_t ready, cudaStream_t built_on, cudaStream_t stream);
 
 // The handle the compute kernels should read: t itself when its widths are 32 or 64 bits,
 // otherwise its (cached) 32-bit shadow.
@@ -161,6 +163,9 @@ enum { SP_PART_MERGE_LAST = 1, SP_PART_MTTKRP = 2, SP_PART_SEGIDS = 3 };
 // (the expanded "outer" index), uint32, cached in the handle.  Needs dims < 2^32.
 sp_status sp_get_segment_ids(sp_tensor* t, cudaStream_t stream, const uint32_t** out);
 sp_status sp_get_merge_partition(sp_tensor* t, int64_t items_per_chunk, cudaStream_t stream, sp_partition* out);
+// Length of the longest last-level segment (row of CSR, stored row of DCSR, ...), measured on the
+// device on first use (one small kernel and one read-back, which waits for the stream) and kept.
+sp_status sp_get_max_segment(sp_tensor* t, cudaStream_t stream, int64_t* out);
 sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t nnz_per_chunk, cudaStream_t stream, sp_partition* out);
 
 // SpMV for rank-2 handles whose inner level is dense (dense_inner.cu).

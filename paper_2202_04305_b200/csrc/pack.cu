@@ -102,10 +102,16 @@ __global__ void k_build_keys(LevelCoords lc, int64_t n, LevelPlan p, uint64_t* k
 }
 
 // ------------------------------------------------------------ radix sort ---
+// Digits are up to kMaxDigitBits wide (512 bins): the 42-bit keys of a 16,384^3 tensor sort in five
+// passes (9, 9, 8, 8, 8 bits).  The kernels are instantiated per digit width so that the ranking
+// needs exactly that many ballots.
+#ifndef SP_SORT_MAX_BITS
+#define SP_SORT_MAX_BITS 9
+#endif
+constexpr int kMaxDigitBits = SP_SORT_MAX_BITS;
 constexpr int kSortThreads = 256;
 constexpr int kSortIpt = 16;
 constexpr int kSortTile = kSortThreads * kSortIpt;   // 4096
-constexpr int kRadix = 256;
 constexpr int kSortWarps = kSortThreads / 32;
 
 __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
@@ -135,13 +141,14 @@ __device__ __forceinline__ uint32_t block256_excl_scan(uint32_t v, uint32_t* sum
     return incl - v + pre;
 }
 
+template <int BITS>
 __global__ void __launch_bounds__(kSortThreads)
-k_sort_upsweep(const uint64_t* __restrict__ keys, int64_t n, int shift, uint32_t mask,
-               uint32_t* __restrict__ tilehist, int64_t ntiles) {
-    __shared__ uint32_t hist[kSortWarps][kRadix];     // one histogram per warp: conflicts only inside a warp
+k_sort_upsweep(const uint64_t* __restrict__ keys, int64_t n, int shift, uint32_t* __restrict__ tilehist, int64_t ntiles) {
+    constexpr int RADIX = 1 << BITS;
+    constexpr uint32_t mask = RADIX - 1;
+    __shared__ uint32_t hist[kSortWarps][RADIX];     // one histogram per warp: conflicts only inside a warp
     const int t = threadIdx.x, w = t >> 5;
-#pragma unroll
-    for (int i = 0; i < kSortWarps; ++i) hist[i][t] = 0;
+    for (int i = t; i < kSortWarps * RADIX; i += kSortThreads) (&hist[0][0])[i] = 0;
     __syncthreads();
     const int64_t base = (int64_t)blockIdx.x * kSortTile;
     uint64_t k[kSortIpt];
@@ -156,21 +163,23 @@ k_sort_upsweep(const uint64_t* __restrict__ keys, int64_t n, int shift, uint32_t
         if (e < n) atomicAdd(&hist[w][(uint32_t)(k[i] >> shift) & mask], 1u);
     }
     __syncthreads();
-    uint32_t c = 0;
+    for (int d = t; d < RADIX; d += kSortThreads) {
+        uint32_t c = 0;
 #pragma unroll
-    for (int i = 0; i < kSortWarps; ++i) c += hist[i][t];
-    tilehist[(int64_t)t * ntiles + blockIdx.x] = c;
+        for (int i = 0; i < kSortWarps; ++i) c += hist[i][d];
+        tilehist[(int64_t)d * ntiles + blockIdx.x] = c;
+    }
 }
 
-// Lanes of the warp whose 9-bit value (digit, or kRadix for padding) equals this lane's, by one
-// ballot per bit.  The hardware match instruction does the same but costs more per call the more
-// distinct values the warp holds: with uniform 8-bit digits the scatter pass ran 0.31 ms per five
-// passes over 5 M entries with it and 0.24 ms with the ballots.  Always nine ballots: stopping at
-// the digit's width through a run-time bound made the loop slower, not faster.
+// Lanes of the warp whose NB-bit value equals this lane's, by one ballot per bit.  The hardware
+// match instruction does the same but costs more per call the more distinct values the warp holds:
+// with uniform 8-bit digits the scatter pass ran 0.31 ms per five passes over 5 M entries with it and
+// 0.24 ms with the ballots.  NB is a compile-time count: a run-time bound made the loop slower.
+template <int NB>
 __device__ __forceinline__ uint32_t same_value_lanes(uint32_t d) {
     uint32_t peers = 0xffffffffu;
 #pragma unroll
-    for (int b = 0; b < 9; ++b) {
+    for (int b = 0; b < NB; ++b) {
         const bool bit = (d >> b) & 1u;
         const uint32_t bal = __ballot_sync(0xffffffffu, bit);
         peers &= bit ? bal : ~bal;
@@ -195,40 +204,65 @@ k_sort_scan(uint32_t* tilehist, int64_t ntiles, uint32_t* digit_total) {
     if (threadIdx.x == 0) digit_total[blockIdx.x] = carry;
 }
 
-constexpr size_t down_smem(bool pay) {
-    return (size_t)kSortTile * 8 + (pay ? (size_t)kSortTile * 4 : 0) + (size_t)kSortWarps * (kRadix + 1) * 4 +
-           (size_t)(kRadix + 1) * 4 + (size_t)kRadix * 8 + 64;
+constexpr size_t down_smem(bool pay, int bits) {
+    return (size_t)kSortTile * 8 + (pay ? (size_t)kSortTile * 4 : 0) + (size_t)kSortWarps * ((1 << bits) + 1) * 4 +
+           (size_t)((1 << bits) + 1) * 4 + (size_t)(1 << bits) * 4 + 64;
+}
+
+// Ranks the warp's 16 rounds of 32 keys: rank i = number of earlier keys of this warp with the same
+// digit (below 512, so two ranks share a register: round i sits in half i & 1 of rank[i / 2]); the
+// per-warp digit counts end up in mycnt[].  NB = BITS, or BITS + 1 when the tile has padding slots
+// (their digit is RADIX, which sorts after every real digit).
+template <int BITS, int NB>
+__device__ __forceinline__ void rank_rounds(const uint64_t (&key)[kSortIpt], int shift, int w, int lane, int tile_n,
+                                            uint32_t* mycnt, uint32_t (&rank)[kSortIpt / 2]) {
+    constexpr uint32_t RADIX = 1u << BITS;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+#pragma unroll
+    for (int i = 0; i < kSortIpt; ++i) {
+        uint32_t d = (uint32_t)(key[i] >> shift) & (RADIX - 1);
+        if (NB > BITS && w * (32 * kSortIpt) + i * 32 + lane >= tile_n) d = RADIX;
+        const uint32_t peers = same_value_lanes<NB>(d);
+        const int leader = __ffs(peers) - 1;
+        uint32_t b = 0;
+        if (lane == leader) { b = mycnt[d]; mycnt[d] = b + (uint32_t)__popc(peers); }
+        b = __shfl_sync(0xffffffffu, b, leader);
+        const uint32_t r = b + (uint32_t)__popc(peers & lt_mask);
+        if (i & 1) rank[i / 2] |= r << 16; else rank[i / 2] = r;
+        __syncwarp();                                 // rounds update the same counters: keep them in order
+    }
 }
 
 // PAY: a 32-bit payload (the entry index) travels beside every key.  Without it the index sits in
 // the key's low bits; the last pass (split_bits >= 0) then separates the two again on the way out:
 // keys_out gets key >> split_bits, idx_out the low split_bits bits.
-template <bool PAY>
+template <bool PAY, int BITS>
 __global__ void __launch_bounds__(kSortThreads, 3)   // three tiles per SM hide the ranking chain's latency
 k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict__ idx_in,
                  uint64_t* __restrict__ keys_out, uint32_t* __restrict__ idx_out, int64_t n, int shift,
-                 uint32_t mask, const uint32_t* __restrict__ tilehist, int64_t ntiles,
+                 const uint32_t* __restrict__ tilehist, int64_t ntiles,
                  const uint32_t* __restrict__ digit_total, int split_bits) {
+    constexpr int RADIX = 1 << BITS;
+    constexpr uint32_t mask = RADIX - 1;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t* skeys = reinterpret_cast<uint64_t*>(smem_raw);
     uint32_t* sidx = reinterpret_cast<uint32_t*>(skeys + kSortTile);
-    uint32_t* wcnt = PAY ? sidx + kSortTile : sidx;           // [warps][kRadix + 1]
-    uint32_t* dstart = wcnt + kSortWarps * (kRadix + 1);      // [kRadix + 1]
-    int64_t* goff = reinterpret_cast<int64_t*>(dstart + (kRadix + 1) + 1);   // [kRadix], 8-byte aligned
+    uint32_t* wcnt = PAY ? sidx + kSortTile : sidx;           // [warps][RADIX + 1]
+    uint32_t* dstart = wcnt + kSortWarps * (RADIX + 1);       // [RADIX + 1]
+    uint32_t* goff = dstart + (RADIX + 1);                    // [RADIX]: global position of the digit's first key minus dstart (mod 2^32)
     __shared__ uint32_t sums[8];
 
     const int t = threadIdx.x, w = t >> 5, lane = t & 31;
     const int64_t base = (int64_t)blockIdx.x * kSortTile;
     const int tile_n = (int)min((int64_t)kSortTile, n - base);
 
-    for (int i = t; i < kSortWarps * (kRadix + 1); i += kSortThreads) wcnt[i] = 0;
+    for (int i = t; i < kSortWarps * (RADIX + 1); i += kSortThreads) wcnt[i] = 0;
     __syncthreads();
 
     uint64_t key[kSortIpt];
     uint32_t pay[kSortIpt];
-    uint32_t rank[kSortIpt];
-    uint32_t* mycnt = wcnt + w * (kRadix + 1);
-    const uint32_t lt_mask = (1u << lane) - 1u;
+    uint32_t rank[kSortIpt / 2];
+    uint32_t* mycnt = wcnt + w * (RADIX + 1);
 #pragma unroll
     for (int i = 0; i < kSortIpt; ++i) {             // all loads first
         const int li = w * (32 * kSortIpt) + i * 32 + lane;
@@ -236,56 +270,63 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
         key[i] = valid ? keys_in[base + li] : 0;
         pay[i] = (PAY && valid) ? idx_in[base + li] : 0;
     }
+    if (tile_n == kSortTile) rank_rounds<BITS, BITS>(key, shift, w, lane, tile_n, mycnt, rank);
+    else rank_rounds<BITS, BITS + 1>(key, shift, w, lane, tile_n, mycnt, rank);
+    __syncthreads();
+
+    // per digit: exclusive scan over warps; then exclusive scan over digits (each thread owns
+    // RADIX / 256 consecutive digits when RADIX > 256)
+    constexpr int DPT = RADIX > kSortThreads ? RADIX / kSortThreads : 1;
+    uint32_t tot_d[DPT], gtot_d[DPT];
+    uint32_t mine = 0, gmine = 0;
+#pragma unroll
+    for (int q = 0; q < DPT; ++q) {
+        const int d = t * DPT + q;
+        tot_d[q] = 0; gtot_d[q] = 0;
+        if (d < RADIX) {
+            uint32_t run = 0;
+            for (int ww = 0; ww < kSortWarps; ++ww) {
+                const uint32_t c = wcnt[ww * (RADIX + 1) + d];
+                wcnt[ww * (RADIX + 1) + d] = run;
+                run += c;
+            }
+            tot_d[q] = run;
+            gtot_d[q] = digit_total[d];
+        }
+        mine += tot_d[q];
+        gmine += gtot_d[q];
+    }
+    if (t == 0) {   // the padding bin: invalid items sort after every real digit
+        uint32_t r2 = 0;
+        for (int ww = 0; ww < kSortWarps; ++ww) {
+            const uint32_t c = wcnt[ww * (RADIX + 1) + RADIX];
+            wcnt[ww * (RADIX + 1) + RADIX] = r2;
+            r2 += c;
+        }
+    }
+    uint32_t tot_all, gtot_all;
+    uint32_t ex = block256_excl_scan(mine, sums, &tot_all);
+    uint32_t gex = block256_excl_scan(gmine, sums, &gtot_all);
+#pragma unroll
+    for (int q = 0; q < DPT; ++q) {
+        const int d = t * DPT + q;
+        if (d < RADIX) {
+            dstart[d] = ex;
+            // global base of digit d = totals of smaller digits + this tile's prefix within the digit
+            goff[d] = gex + tilehist[(int64_t)d * ntiles + blockIdx.x] - ex;
+            ex += tot_d[q];
+            gex += gtot_d[q];
+        }
+    }
+    if (t == 0) dstart[RADIX] = tot_all;
+    __syncthreads();
+
 #pragma unroll
     for (int i = 0; i < kSortIpt; ++i) {
         const int li = w * (32 * kSortIpt) + i * 32 + lane;
-        const uint32_t d = li < tile_n ? ((uint32_t)(key[i] >> shift) & mask) : (uint32_t)kRadix;
-        const uint32_t peers = same_value_lanes(d);
-        const int leader = __ffs(peers) - 1;
-        uint32_t b = 0;
-        if (lane == leader) { b = mycnt[d]; mycnt[d] = b + (uint32_t)__popc(peers); }
-        b = __shfl_sync(0xffffffffu, b, leader);
-        rank[i] = b + (uint32_t)__popc(peers & lt_mask);
-        __syncwarp();                                 // rounds update the same counters: keep them in order
-    }
-    __syncthreads();
-
-    // per digit: exclusive scan over warps; then exclusive scan over digits
-    uint32_t total = 0;
-    {
-        uint32_t run = 0;
-        for (int ww = 0; ww < kSortWarps; ++ww) {
-            uint32_t c = wcnt[ww * (kRadix + 1) + t];
-            wcnt[ww * (kRadix + 1) + t] = run;
-            run += c;
-        }
-        total = run;
-        if (t == 0) {   // the padding bin: invalid items sort after every real digit
-            uint32_t r2 = 0;
-            for (int ww = 0; ww < kSortWarps; ++ww) {
-                uint32_t c = wcnt[ww * (kRadix + 1) + kRadix];
-                wcnt[ww * (kRadix + 1) + kRadix] = r2;
-                r2 += c;
-            }
-        }
-    }
-    uint32_t tot_all;
-    uint32_t ex = block256_excl_scan(total, sums, &tot_all);
-    dstart[t] = ex;
-    if (t == 0) dstart[kRadix] = tot_all;
-    // global base of digit t = sum of totals of smaller digits + this tile's prefix within the digit
-    uint32_t dt = digit_total[t];
-    uint32_t gtot;
-    uint32_t gex = block256_excl_scan(dt, sums, &gtot);
-    goff[t] = (int64_t)gex + (int64_t)tilehist[(int64_t)t * ntiles + blockIdx.x] - (int64_t)ex;
-    __syncthreads();
-
-#pragma unroll
-    for (int i = 0; i < kSortIpt; ++i) {
-        int li = w * (32 * kSortIpt) + i * 32 + lane;
-        bool valid = li < tile_n;
-        uint32_t d = valid ? ((uint32_t)(key[i] >> shift) & mask) : (uint32_t)kRadix;
-        uint32_t s = dstart[d] + mycnt[d] + rank[i];
+        const bool valid = li < tile_n;
+        const uint32_t d = valid ? ((uint32_t)(key[i] >> shift) & mask) : (uint32_t)RADIX;
+        const uint32_t s = dstart[d] + mycnt[d] + ((i & 1) ? rank[i / 2] >> 16 : rank[i / 2] & 0xffffu);
         if (valid) {
             skeys[s] = key[i];
             if (PAY) sidx[s] = pay[i];
@@ -293,9 +334,9 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
     }
     __syncthreads();
     for (int s = t; s < tile_n; s += kSortThreads) {
-        uint64_t k = skeys[s];
-        uint32_t d = (uint32_t)(k >> shift) & mask;
-        int64_t o = goff[d] + s;
+        const uint64_t k = skeys[s];
+        const uint32_t d = (uint32_t)(k >> shift) & mask;
+        const uint32_t o = goff[d] + (uint32_t)s;
         if (PAY) {
             keys_out[o] = k;
             idx_out[o] = sidx[s];
@@ -306,6 +347,32 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
             keys_out[o] = k;
         }
     }
+}
+
+// One radix pass (histograms, per-digit scans, ranked scatter) for a digit of `bits` bits at `shift`.
+template <int BITS>
+sp_status sort_pass(const uint64_t* kin, const uint32_t* iin, uint64_t* kout, uint32_t* iout, int64_t n, int shift,
+                    uint32_t* tilehist, int64_t stiles, uint32_t* digit_total, bool fused, int split_bits,
+                    cudaStream_t stream, PhaseTimer& timer) {
+    k_sort_upsweep<BITS><<<(unsigned)stiles, kSortThreads, 0, stream>>>(kin, n, shift, tilehist, stiles);
+    timer.mark(kPhUpsweep);
+    k_sort_scan<<<1 << BITS, 256, 0, stream>>>(tilehist, stiles, digit_total);
+    timer.mark(kPhScan);
+    if (fused) {
+        SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep<false, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)down_smem(false, BITS)));
+        k_sort_downsweep<false, BITS><<<(unsigned)stiles, kSortThreads, down_smem(false, BITS), stream>>>(
+            kin, nullptr, kout, iout, n, shift, tilehist, stiles, digit_total, split_bits);
+    } else {
+        SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep<true, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)down_smem(true, BITS)));
+        k_sort_downsweep<true, BITS><<<(unsigned)stiles, kSortThreads, down_smem(true, BITS), stream>>>(
+            kin, iin, kout, iout, n, shift, tilehist, stiles, digit_total, -1);
+    }
+    SP_LAUNCH_CHECK();
+    timer.mark(kPhDownsweep);
+    sp_count_launches(3);
+    return SP_OK;
 }
 
 // ------------------------------------------------- flags, counts, emit ---
@@ -694,8 +761,8 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         uint32_t* ibuf[2] = {ws.get<uint32_t>((size_t)n), ws.get<uint32_t>((size_t)n)};
         d_err = ws.get<int>(1);
         const int64_t stiles = sp_ceil_div(n, kSortTile);
-        uint32_t* tilehist = ws.get<uint32_t>((size_t)stiles * kRadix);
-        uint32_t* digit_total = ws.get<uint32_t>(kRadix);
+        uint32_t* tilehist = ws.get<uint32_t>((size_t)stiles << kMaxDigitBits);
+        uint32_t* digit_total = ws.get<uint32_t>((size_t)1 << kMaxDigitBits);
         ct_tiles = sp_ceil_div(n, kCtTile);
         uint64_t* tilesum = ws.get<uint64_t>((size_t)ct_tiles);
         tileprefix = ws.get<int64_t>((size_t)ct_tiles * SP_MAX_RANK);
@@ -705,7 +772,7 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
 
         LevelCoords lc;
         for (int l = 0; l < SP_MAX_RANK; ++l) lc.p[l] = coo_coords[l < rank ? plan.src[l] : 0];
-        const int npasses = (total_bits + 7) / 8;
+        const int npasses = (total_bits + kMaxDigitBits - 1) / kMaxDigitBits;
         // the entry index rides inside the key when both fit in 64 bits
         int idx_bits = 0;
         while (((int64_t)1 << idx_bits) < n) ++idx_bits;
@@ -718,29 +785,29 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         SP_LAUNCH_CHECK();
         sp_count_launches(1);
         timer.mark(kPhKeys);
-        SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)down_smem(true)));
-        SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)down_smem(false)));
-        const int per = npasses ? (total_bits + npasses - 1) / npasses : 0;
-        int cur = 0;
+        // digit widths as even as possible, the wider ones first (42 bits: 9, 9, 8, 8, 8)
+        int cur = 0, kshift = 0;
         for (int ps = 0; ps < npasses; ++ps) {
-            const int kshift = ps * per;                     // position of the digit inside the level key
-            const int width = (kshift + per <= total_bits) ? per : (total_bits - kshift);
+            const int left = npasses - ps;
+            const int width = (total_bits - kshift + left - 1) / left;
             const int shift = kshift + (fused ? idx_bits : 0);
-            const uint32_t mask = (1u << width) - 1u;
-            k_sort_upsweep<<<(unsigned)stiles, kSortThreads, 0, stream>>>(kbuf[cur], n, shift, mask, tilehist, stiles);
-            timer.mark(kPhUpsweep);
-            k_sort_scan<<<kRadix, 256, 0, stream>>>(tilehist, stiles, digit_total);
-            timer.mark(kPhScan);
-            if (fused)
-                k_sort_downsweep<false><<<(unsigned)stiles, kSortThreads, down_smem(false), stream>>>(
-                    kbuf[cur], nullptr, kbuf[cur ^ 1], ibuf[cur ^ 1], n, shift, mask, tilehist, stiles, digit_total,
-                    ps == npasses - 1 ? idx_bits : -1);
-            else
-                k_sort_downsweep<true><<<(unsigned)stiles, kSortThreads, down_smem(true), stream>>>(
-                    kbuf[cur], ibuf[cur], kbuf[cur ^ 1], ibuf[cur ^ 1], n, shift, mask, tilehist, stiles, digit_total, -1);
-            SP_LAUNCH_CHECK();
-            timer.mark(kPhDownsweep);
-            sp_count_launches(3);
+            const int split = (fused && ps == npasses - 1) ? idx_bits : -1;
+            sp_status ps_st = SP_ERR_UNSUPPORTED;
+#define SP_SORT_PASS(B)                                                                                             \
+    case B:                                                                                                         \
+        ps_st = sort_pass<B>(kbuf[cur], ibuf[cur], kbuf[cur ^ 1], ibuf[cur ^ 1], n, shift, tilehist, stiles,        \
+                             digit_total, fused, split, stream, timer);                                             \
+        break;
+            switch (width) {
+                SP_SORT_PASS(1) SP_SORT_PASS(2) SP_SORT_PASS(3) SP_SORT_PASS(4) SP_SORT_PASS(5)
+                SP_SORT_PASS(6) SP_SORT_PASS(7) SP_SORT_PASS(8)
+#if SP_SORT_MAX_BITS >= 9
+                SP_SORT_PASS(9)
+#endif
+            }
+#undef SP_SORT_PASS
+            if (ps_st != SP_OK) return ps_st;
+            kshift += width;
             cur ^= 1;
         }
         npasses_done = npasses;

@@ -61,7 +61,46 @@ __global__ void k_segment_ids(const P* __restrict__ pos, int64_t nseg, int64_t n
     seg[p] = outer ? (uint32_t)outer[lo] : (uint32_t)lo;
 }
 
+// Longest segment: grid-stride maximum of pos[q+1] - pos[q], one atomicMax per block.
+template <typename P>
+__global__ void k_max_segment(const P* __restrict__ pos, int64_t nseg, unsigned long long* __restrict__ out) {
+    unsigned long long m = 0;
+    for (int64_t q = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; q < nseg; q += (int64_t)gridDim.x * blockDim.x) {
+        const unsigned long long len = (unsigned long long)pos[q + 1] - (unsigned long long)pos[q];
+        m = len > m ? len : m;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long u = __shfl_xor_sync(0xffffffffu, m, o);
+        m = u > m ? u : m;
+    }
+    if ((threadIdx.x & 31) == 0 && m > 0) atomicMax(out, m);
+}
+
 }  // namespace
+
+sp_status sp_get_max_segment(sp_tensor* t, cudaStream_t stream, int64_t* out) {
+    std::lock_guard<std::mutex> lock(t->mu);
+    if (t->max_seg >= 0) { *out = t->max_seg; return SP_OK; }
+    const int last = t->rank - 1;
+    const int64_t nseg = t->npos[last] - 1;
+    if (nseg <= 0 || t->ncrd[last] == 0) { t->max_seg = 0; *out = 0; return SP_OK; }
+    sp_workspace ws(stream);
+    unsigned long long* d = ws.get<unsigned long long>(1);
+    if (ws.failed) return SP_ERR_ALLOC;
+    SP_CUDA(cudaMemsetAsync(d, 0, sizeof *d, stream));
+    const unsigned blocks = (unsigned)std::min<int64_t>(sp_ceil_div(nseg, 256), 148 * 8);
+    if (t->posBits == 32) k_max_segment<uint32_t><<<blocks, 256, 0, stream>>>(static_cast<const uint32_t*>(t->pos[last]), nseg, d);
+    else k_max_segment<uint64_t><<<blocks, 256, 0, stream>>>(static_cast<const uint64_t*>(t->pos[last]), nseg, d);
+    SP_LAUNCH_CHECK();
+    sp_count_launches(1);
+    unsigned long long h = 0;
+    SP_CUDA(cudaMemcpyAsync(&h, d, sizeof h, cudaMemcpyDeviceToHost, stream));
+    SP_CUDA(cudaStreamSynchronize(stream));
+    t->max_seg = (int64_t)h;
+    *out = t->max_seg;
+    return SP_OK;
+}
 
 sp_status sp_get_segment_ids(sp_tensor* t, cudaStream_t stream, const uint32_t** out) {
     std::lock_guard<std::mutex> lock(t->mu);
@@ -157,8 +196,7 @@ sp_status sp_widened(sp_tensor* t, cudaStream_t stream, sp_tensor** out) {
     std::lock_guard<std::mutex> lock(t->mu);
     if (t->wide) {
         *out = t->wide;
-        if (t->wide_ready && stream != t->wide_built_on) SP_CUDA(cudaStreamWaitEvent(stream, t->wide_ready, 0));
-        return SP_OK;
+        return sp_event_wait(t->wide_ready, t->wide_built_on, stream);
     }
     sp_tensor* w = new sp_tensor();
     w->rank = t->rank;

@@ -178,6 +178,40 @@ __global__ void k_spmv_fixup(const double* __restrict__ carry_val, const int64_t
     y[outer ? (int64_t)outer[r] : r] += s;
 }
 
+// Row-major SpMV for matrices of short rows: G lanes per stored row, no staging, no carries.
+// Every lane issues its (up to four) coordinate and value loads, then the gathered x entries,
+// before the first multiply-add; the row's sum is folded over the group's lanes and written once.
+// Rows without entries (CSR) are written as zeros here; rows that DCSR elides were zeroed before.
+template <typename P, typename I, int G>
+__global__ void __launch_bounds__(256)
+k_spmv_rows(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
+            const I* __restrict__ outer, const double* __restrict__ x, double* __restrict__ y, int64_t nseg) {
+    constexpr int kU = 4;
+    const int64_t q = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) / G;
+    const int gl = threadIdx.x % G;
+    const bool live = q < nseg;
+    const int64_t p0 = live ? (int64_t)pos[q] : 0, p1 = live ? (int64_t)pos[q + 1] : 0;
+    double s = 0.0;
+    for (int64_t p = p0 + gl; p < p1; p += kU * G) {
+        I c[kU];
+        double v[kU], xx[kU];
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int64_t pp = p + u * G;
+            const bool ok = pp < p1;
+            c[u] = ok ? crd[pp] : (I)0;
+            v[u] = ok ? val[pp] : 0.0;
+        }
+#pragma unroll
+        for (int u = 0; u < kU; ++u) xx[u] = (p + u * G < p1) ? __ldg(x + c[u]) : 0.0;
+#pragma unroll
+        for (int u = 0; u < kU; ++u) s = fma(v[u], xx[u], s);
+    }
+#pragma unroll
+    for (int o = G / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (live && gl == 0) y[outer ? (int64_t)outer[q] : q] = s;
+}
+
 // ===================================================================== SpMM
 constexpr int kMThreads = 256;
 constexpr int kMItems = 128;   // merge items per warp
@@ -398,6 +432,31 @@ extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* str
     if (!rowmajor || dbl) SP_CUDA(cudaMemsetAsync(y, 0, (size_t)m * sizeof(double), stream));
     const int64_t nseg = A->npos[1] - 1;
     if (nseg <= 0) return SP_OK;
+    // Short rows (mean <= 64 entries, none longer than 4096): a lane group per row, one launch.
+    // Anything skewed or long goes through the merge path below, whose cost does not depend on the
+    // row lengths.
+    if (rowmajor && A->ncrd[1] <= 64 * nseg) {
+        int64_t max_seg = 0;
+        const sp_status ms = sp_get_max_segment(A, stream, &max_seg);
+        if (ms != SP_OK) return ms;
+        if (max_seg <= 4096) {
+            const int64_t mean = A->ncrd[1] / nseg;
+            const int G = mean <= 6 ? 4 : (mean <= 12 ? 8 : (mean <= 24 ? 16 : 32));
+            const unsigned blocks = (unsigned)sp_ceil_div(nseg * G, 256);
+            SP_DISPATCH_WIDTHS(A, {
+                const P* pos = static_cast<const P*>(A->pos[1]);
+                const I* crd = static_cast<const I*>(A->crd[1]);
+                const I* outer = dbl ? static_cast<const I*>(A->crd[0]) : nullptr;
+                if (G == 4) k_spmv_rows<P, I, 4><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg);
+                else if (G == 8) k_spmv_rows<P, I, 8><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg);
+                else if (G == 16) k_spmv_rows<P, I, 16><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg);
+                else k_spmv_rows<P, I, 32><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg);
+            });
+            SP_LAUNCH_CHECK();
+            sp_count_launches(1);
+            return SP_OK;
+        }
+    }
     sp_partition part;
     sp_status st = sp_get_merge_partition(A, kVTile, stream, &part);
     if (st != SP_OK) return st;
