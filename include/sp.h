@@ -28,8 +28,9 @@
  *     An encoding a kernel does not handle yields SP_ERR_UNSUPPORTED, never a
  *     different algorithm on the host.
  *   - A handle is immutable after sp_pack.  Kernels cache read-only work-partition
- *     tables inside it on first use (under the handle's lock; a call on another
- *     stream waits for the stream that built them); everything a call writes
+ *     tables inside it on first use (under the handle's lock; that first call
+ *     waits for the stream once, so the tables are complete for every stream
+ *     afterwards); everything a call writes
  *     besides its output is scratch it takes from the allocator for that call, so
  *     calls on different streams or host threads may share a handle.  The handle
  *     must be used with the device it was packed on current

@@ -16,7 +16,11 @@ MAX_RANK = 5
 DUP_SUM, DUP_ERROR = 0, 1
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libsp.so")
+# SP_DEBUG_BOUNDS=1 in the environment selects the bounds-checking build of the same library (every
+# index derived from stored positions / coordinates is checked on the device; a bad one makes the call
+# return SP_ERR_OUT_OF_RANGE instead of reading or writing out of bounds).  Much slower; for debugging.
+DEBUG_BOUNDS = os.environ.get("SP_DEBUG_BOUNDS", "") not in ("", "0")
+_LIB_PATH = os.path.join(_HERE, "libsp_debug_bounds.so" if DEBUG_BOUNDS else "libsp.so")
 
 SYMBOLS = ["sp_status_string", "sp_set_allocator", "sp_pack", "sp_free", "sp_info", "sp_positions",
            "sp_coordinates", "sp_values", "sp_unpack", "sp_spmv", "sp_spmm", "sp_sddmm", "sp_mttkrp",
@@ -32,8 +36,8 @@ class SpError(RuntimeError):
 
 def _load():
     if not os.path.exists(_LIB_PATH):
-        raise ImportError(f"{_LIB_PATH} not found: build it with `python -m paper_2202_04305_b200.build` "
-                          "(there is no CPU fallback)")
+        raise ImportError(f"{_LIB_PATH} not found: build it with `python -m paper_2202_04305_b200.build"
+                          f"{' --debug-bounds' if DEBUG_BOUNDS else ''}` (there is no CPU fallback)")
     lib = C.CDLL(_LIB_PATH)
     lib.sp_status_string.restype = C.c_char_p
     lib.sp_status_string.argtypes = [C.c_int]

@@ -31,12 +31,12 @@ def _newest_header() -> float:
     return max(os.path.getmtime(h) for h in hs)
 
 
-def _compile(src: str, verbose: bool) -> str:
+def _compile(src: str, verbose: bool, obj_dir: str = OBJ, extra=()) -> str:
     s = os.path.join(CSRC, src)
-    o = os.path.join(OBJ, src.replace(".cu", ".o"))
+    o = os.path.join(obj_dir, src.replace(".cu", ".o"))
     if os.path.exists(o) and os.path.getmtime(o) >= max(os.path.getmtime(s), _newest_header()):
         return o
-    cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
+    cmd = [_nvcc()] + NVCC_FLAGS + list(extra) + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or r.returncode:
         sys.stderr.write(r.stdout + r.stderr)
@@ -45,17 +45,25 @@ def _compile(src: str, verbose: bool) -> str:
     return o
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    os.makedirs(OBJ, exist_ok=True)
+LIB_DEBUG = os.path.join(HERE, "libsp_debug_bounds.so")
+
+
+def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False) -> str:
+    """debug_bounds: the checking build (-DSP_DEBUG_BOUNDS, see csrc/common.cuh) as a second library,
+    libsp_debug_bounds.so, with its own object folder; the normal library is untouched."""
+    obj_dir = OBJ + "_debug_bounds" if debug_bounds else OBJ
+    lib = LIB_DEBUG if debug_bounds else LIB
+    extra = ("-DSP_DEBUG_BOUNDS",) if debug_bounds else ()
+    os.makedirs(obj_dir, exist_ok=True)
     if force:
-        for f in os.listdir(OBJ):
-            os.remove(os.path.join(OBJ, f))
+        for f in os.listdir(obj_dir):
+            os.remove(os.path.join(obj_dir, f))
     with cf.ThreadPoolExecutor(max_workers=8) as ex:
-        objs = list(ex.map(lambda s: _compile(s, verbose), SOURCES))
-    if force or not os.path.exists(LIB) or any(os.path.getmtime(o) > os.path.getmtime(LIB) for o in objs):
-        subprocess.check_call([_nvcc(), "-Wno-deprecated-gpu-targets", "-shared", "-o", LIB] + objs + ["-lcudart"])
-    return LIB
+        objs = list(ex.map(lambda s: _compile(s, verbose, obj_dir, extra), SOURCES))
+    if force or not os.path.exists(lib) or any(os.path.getmtime(o) > os.path.getmtime(lib) for o in objs):
+        subprocess.check_call([_nvcc(), "-Wno-deprecated-gpu-targets", "-shared", "-o", lib] + objs + ["-lcudart"])
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug_bounds="--debug-bounds" in sys.argv))

@@ -34,29 +34,9 @@ sp_status sp_check_device(const sp_tensor* t) {
     return dev == t->device ? SP_OK : SP_ERR_INVALID_ARG;
 }
 
-sp_status sp_partition_built(sp_partition* p, cudaStream_t stream) {
-    SP_CUDA(cudaEventCreateWithFlags(&p->ready, cudaEventDisableTiming));
-    SP_CUDA(cudaEventRecord(p->ready, stream));
-    p->built_on = stream;
+sp_status sp_partition_built(cudaStream_t stream) {
+    SP_CUDA(cudaStreamSynchronize(stream));
     return SP_OK;
-}
-
-sp_status sp_event_wait(cudaEvent_t ready, cudaStream_t built_on, cudaStream_t stream) {
-    if (!ready || stream == built_on) return SP_OK;
-    const cudaError_t q = cudaEventQuery(ready);
-    if (q == cudaSuccess) return SP_OK;                 // the table was finished long ago: nothing to wait for
-    if (q != cudaErrorNotReady) { cudaGetLastError(); return SP_ERR_CUDA; }
-    cudaGetLastError();
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    SP_CUDA(cudaStreamIsCapturing(stream, &cap));
-    // a stream that is being captured cannot wait for work outside its graph: finish that work first
-    if (cap != cudaStreamCaptureStatusNone) SP_CUDA(cudaEventSynchronize(ready));
-    else SP_CUDA(cudaStreamWaitEvent(stream, ready, 0));
-    return SP_OK;
-}
-
-sp_status sp_partition_wait(const sp_partition& p, cudaStream_t stream) {
-    return sp_event_wait(p.ready, p.built_on, stream);
 }
 
 extern "C" {
@@ -98,12 +78,10 @@ sp_status sp_free(sp_tensor* t) {
     }
     if (t->owns_val) sp_dev_free(t->val, nullptr);
     if (t->wide) sp_free(t->wide);
-    if (t->wide_ready) cudaEventDestroy(t->wide_ready);
     for (auto& kv : t->parts) {
         sp_dev_free(kv.second.row, nullptr);
         sp_dev_free(kv.second.nz, nullptr);
         sp_dev_free(kv.second.aux, nullptr);
-        if (kv.second.ready) cudaEventDestroy(kv.second.ready);
     }
     delete t;
     cudaSetDevice(prev);

@@ -15,18 +15,16 @@
 // ---------------------------------------------------------------------------
 
 // Work-partition table cached in a handle: chunk w covers merge-path
-// coordinates [(row[w], nz[w]), (row[w+1], nz[w+1])).  The arrays are written once, by the
-// kernels enqueued on `built_on` when the table is created, and only read afterwards; `ready`
-// marks the end of that work so that a call on another stream can wait for it.  Scratch that a
-// call writes (row carries) is never kept here: every call takes its own from the allocator, so
-// calls on different streams share nothing writable.
+// coordinates [(row[w], nz[w]), (row[w+1], nz[w+1])).  The arrays are written once, when the table
+// is created (the creating call waits for that work before it publishes the table, so any stream
+// may read it afterwards), and only read from then on.  Scratch that a call writes (row carries)
+// is never kept here: every call takes its own from the allocator, so calls on different streams
+// share nothing writable.
 struct sp_partition {
     int64_t nchunks = 0;
     int64_t* row = nullptr;   // nchunks + 1 entries (device)
     int64_t* nz = nullptr;    // nchunks + 1 entries (device)
     int64_t* aux = nullptr;   // kernel-specific (MTTKRP: slice of each chunk start)
-    cudaEvent_t ready = nullptr;
-    cudaStream_t built_on = nullptr;
 };
 
 struct sp_tensor {
@@ -49,18 +47,13 @@ struct sp_tensor {
     // first use by sp_widened(), owned by this handle.
     int64_t max_seg = -1;      // longest segment of the last level (entries under one parent); -1 = not measured yet
     sp_tensor* wide = nullptr;
-    cudaEvent_t wide_ready = nullptr;
-    cudaStream_t wide_built_on = nullptr;
     bool owns_val = true;
 };
 
 // SP_ERR_INVALID_ARG unless the handle's arrays live on the current device.
 sp_status sp_check_device(const sp_tensor* t);
-// Marks the end of the work that fills a cached table (p->ready, p->built_on).
-sp_status sp_partition_built(sp_partition* p, cudaStream_t stream);
-// Makes `stream` wait for that work when it is not the stream that did it (and it is still running).
-sp_status sp_partition_wait(const sp_partition& p, cudaStream_t stream);
-sp_status sp_event_wait(cudaEvent_t ready, cudaStream_t built_on, cudaStream_t stream);
+// Waits for the work that fills a cached table, so that the table can be published to every stream.
+sp_status sp_partition_built(cudaStream_t stream);
 
 // The handle the compute kernels should read: t itself when its widths are 32 or 64 bits,
 // otherwise its (cached) 32-bit shadow.
@@ -142,11 +135,42 @@ __device__ __forceinline__ void sp_store_uint(void* base, int64_t i, uint64_t v,
 
 __device__ __forceinline__ unsigned sp_lane() { return threadIdx.x & 31u; }
 
+// Debug build (-DSP_DEBUG_BOUNDS): every index that a kernel derives from stored positions or
+// coordinates is checked against the array it addresses.  A bad index is recorded (source line of the
+// check, in this translation unit's device word) and replaced by a valid one, so the kernel finishes
+// without a fault; the API call then reads the word back and returns SP_ERR_OUT_OF_RANGE.  In the
+// normal build SP_IDX(i, n) is just i.
+#ifdef SP_DEBUG_BOUNDS
+static __device__ unsigned long long sp_bounds_word = 0;
+__device__ __forceinline__ int64_t sp_checked_index(int64_t i, int64_t n, int line) {
+    if (i >= 0 && i < n) return i;
+    atomicMax(&sp_bounds_word, ((unsigned long long)line << 32) | 1ull);
+    return (n > 0 && i >= n) ? n - 1 : 0;
+}
+#define SP_IDX(i, n) sp_checked_index((int64_t)(i), (int64_t)(n), __LINE__)
+#else
+#define SP_IDX(i, n) (i)
+#endif
+
 __device__ __forceinline__ double sp_shfl(double v, int src) {
     return __shfl_sync(0xffffffffu, v, src);
 }
 
 #endif  // __CUDACC__
+
+#if defined(SP_DEBUG_BOUNDS) && defined(__CUDACC__)
+// Host side of the debug build: waits for the stream, reads and clears this translation unit's word.
+static inline sp_status sp_bounds_result(cudaStream_t stream) {
+    unsigned long long w = 0, zero = 0;
+    SP_CUDA(cudaStreamSynchronize(stream));
+    SP_CUDA(cudaMemcpyFromSymbol(&w, sp_bounds_word, sizeof w));
+    if (w) SP_CUDA(cudaMemcpyToSymbol(sp_bounds_word, &zero, sizeof zero));
+    return w ? SP_ERR_OUT_OF_RANGE : SP_OK;
+}
+#define SP_BOUNDS_RETURN(stream) do { const sp_status b__ = sp_bounds_result(stream); if (b__ != SP_OK) return b__; } while (0)
+#else
+#define SP_BOUNDS_RETURN(stream) do {} while (0)
+#endif
 
 // Calls f(P{}, I{}) with the unsigned types matching the handle's widths.
 #define SP_DISPATCH_WIDTHS(t, ...)                                              \

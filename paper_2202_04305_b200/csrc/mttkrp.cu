@@ -33,7 +33,8 @@ k_mttkrp(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* __rest
          const I* __restrict__ crd1, const I* __restrict__ crd2, const double* __restrict__ val,
          const double* __restrict__ F1, const double* __restrict__ F2, int64_t R, double* __restrict__ M,
          const int64_t* __restrict__ pfiber, const int64_t* __restrict__ pnz, const int64_t* __restrict__ pslice,
-         int64_t nchunks, int64_t nslice, int64_t nfiber) {
+         int64_t nchunks, int64_t nslice, int64_t nfiber, int64_t d0, int64_t d1, int64_t d2) {
+    // d0, d1, d2: rows of M, F1, F2 (used by the bounds-checking debug build only)
     // open-slice sums of the block's warps: slot 2*warp = the slice the warp's range starts in,
     // slot 2*warp+1 = the slice it ends in (when different); equal neighbours are added here so
     // that a slice spanning the whole block costs one atomic add per column, not one per warp
@@ -80,11 +81,11 @@ k_mttkrp(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* __rest
                         const int t = g * kGroup + u;
                         c[u] = 0.0; b[u] = 0.0;
                         if (t < cnt) {
-                            const int64_t k = (int64_t)__shfl_sync(0xffffffffu, k_l, t);
+                            const int64_t k = SP_IDX(__shfl_sync(0xffffffffu, k_l, t), d2);
                             c[u] = F2r[k * R];
                             if ((endmask >> t) & 1u) {
                                 const int fi = fi0 + __popc(endmask & ((1u << t) - 1u));
-                                const int64_t j = (int64_t)__shfl_sync(0xffffffffu, j_l, fi);
+                                const int64_t j = SP_IDX(__shfl_sync(0xffffffffu, j_l, fi), d1);
                                 b[u] = F1r[j * R];
                             }
                         }
@@ -100,7 +101,7 @@ k_mttkrp(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* __rest
                                 accf = 0.0;
                                 ++f;
                                 if (f == send) {                    // and so is the slice
-                                    const int64_t i = crd0 ? (int64_t)crd0[s] : s;
+                                    const int64_t i = SP_IDX(crd0 ? (int64_t)crd0[s] : s, d0);
                                     if (first) { head_id = i; head_v = accs; }
                                     else if (on) M[i * R + r] = accs;
                                     first = false;
@@ -124,10 +125,10 @@ k_mttkrp(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* __rest
         }
         if (p1 > last_flush) {                      // the range ends inside slice s
             if (f < nfiber && (int64_t)pos2[f] < p1) {   // ... and inside fibre f
-                const double bj = F1r[(int64_t)crd1[f] * R];
+                const double bj = F1r[SP_IDX(crd1[f], d1) * R];
                 accs = fma(bj, accf, accs);
             }
-            const int64_t i = crd0 ? (int64_t)crd0[s] : s;
+            const int64_t i = SP_IDX(crd0 ? (int64_t)crd0[s] : s, d0);
             if (first) { head_id = i; head_v = accs; }
             else { tail_id = i; tail_v = accs; }
         }
@@ -197,12 +198,14 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
               const I* __restrict__ crd1, const I* __restrict__ crd2, const double* __restrict__ val,
               const double* __restrict__ F1, const double* __restrict__ F2, int64_t R, double* __restrict__ M,
               const int64_t* __restrict__ pfiber, const int64_t* __restrict__ pnz,
-              const int64_t* __restrict__ pslice, int64_t nchunks, int64_t nslice, int64_t nfiber) {
+              const int64_t* __restrict__ pslice, int64_t nchunks, int64_t nslice, int64_t nfiber,
+              int64_t d0, int64_t d1, int64_t d2) {
     constexpr int GL = 32 / S;      // lanes per group = entries per group and batch
     constexpr int kStepGroup = S == 2 ? 4 : 2;
-    __shared__ Staged s_st[kTThreads / 32][32];
-    __shared__ double s_car[2 * kTThreads / 32][32];
-    __shared__ long long s_id[2 * kTThreads / 32];
+    constexpr int kWarps = kTThreads / 32;
+    __shared__ Staged s_st[kWarps][32];
+    __shared__ double s_car[2 * kWarps][32];
+    __shared__ long long s_id[2 * kWarps];
     const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5, g = lane / GL, hl = lane % GL;
     const bool live = w < nchunks;
@@ -239,7 +242,7 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
             if (fb + 32 + lane < nfiber) { feB = (int64_t)pos2[fb + 32 + lane + 1]; jB = crd1[fb + 32 + lane]; }
             if (fb + 64 + lane < nfiber) { feC = (int64_t)pos2[fb + 64 + lane + 1]; jC = crd1[fb + 64 + lane]; }
         }
-        I k_n = (p + lane < p1) ? crd2[p + lane] : (I)0;
+        uint32_t k_n = (p + lane < p1) ? (uint32_t)crd2[p + lane] : 0u;
         double v_n = (p + lane < p1) ? val[p + lane] : 0.0;
 
         auto fold_groups = [&]() {       // add the S groups' slice sums into group 0's lanes
@@ -253,11 +256,11 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
             int64_t lim = p1 - p;
             if (slice_end - p < lim) lim = slice_end - p;
             const int cnt = lim < 32 ? (int)lim : 32;
-            const I k_l = k_n;
+            const uint32_t k_l = k_n;
             const double v_l = v_n;
             {
                 const int64_t pn = p + cnt;
-                k_n = (pn + lane < p1) ? crd2[pn + lane] : (I)0;
+                k_n = (pn + lane < p1) ? (uint32_t)crd2[pn + lane] : 0u;
                 v_n = (pn + lane < p1) ? val[pn + lane] : 0.0;
             }
             const int64_t relA = feA - p - 1, relB = feB - p - 1;
@@ -267,11 +270,11 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
             const int fi = (int)(f - fb) + __popc(endmask & ((1u << lane) - 1u));
             const I ja = __shfl_sync(0xffffffffu, jA, fi & 31);
             const I jb = __shfl_sync(0xffffffffu, jB, fi & 31);
-            const uint32_t j = (uint32_t)(fi < 32 ? ja : jb);
+            const uint32_t j = (uint32_t)SP_IDX(fi < 32 ? ja : jb, d1);
             const bool valid = lane < cnt;
             const bool close = valid && (((endmask >> lane) & 1u) || lane == cnt - 1 || hl == GL - 1);
             Staged st;
-            st.koff = valid ? (uint32_t)k_l * Ru : 0u;
+            st.koff = valid ? (uint32_t)SP_IDX(k_l, d2) * Ru : 0u;
             st.bw = valid ? (((j * Ru) << 1) | (close ? 1u : 0u)) : 0u;
             st.v = valid ? v_l : 0.0;
             s_st[wi][lane] = st;
@@ -312,7 +315,7 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
             p += cnt;
             if (p == slice_end) {                    // slice s is complete: all groups' sums -> row i
                 fold_groups();
-                const int64_t i = crd0 ? (int64_t)crd0[s] : s;
+                const int64_t i = SP_IDX(crd0 ? (int64_t)crd0[s] : s, d0);
                 if (first) {
                     head_id = i;
 #pragma unroll
@@ -341,7 +344,7 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
         }
         if (p1 > last_flush) {                       // the range ends inside slice s
             fold_groups();
-            const int64_t i = crd0 ? (int64_t)crd0[s] : s;
+            const int64_t i = SP_IDX(crd0 ? (int64_t)crd0[s] : s, d0);
             if (first) {
                 head_id = i;
 #pragma unroll
@@ -362,7 +365,7 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
         }
         if (lane == 0) { s_id[2 * wi] = head_id; s_id[2 * wi + 1] = tail_id; }
         __syncthreads();
-        constexpr int kSlots = 2 * kTThreads / 32;
+        constexpr int kSlots = 2 * kWarps;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int e = 2 * wi + h;
@@ -435,22 +438,25 @@ static sp_status mttkrp_levels(sp_tensor* T, const double* F1, const double* F2,
     k_mttkrp_fast<P, I, S><<<blocks, kTThreads, 0, stream>>>(                                                          \
         static_cast<const P*>(T->pos[1]), T->lt[0] == SP_COMPRESSED ? static_cast<const I*>(T->crd[0]) : nullptr,      \
         static_cast<const P*>(T->pos[2]), static_cast<const I*>(T->crd[1]), static_cast<const I*>(T->crd[2]), T->val,  \
-        F1, F2, R, M, part.row, part.nz, part.aux, part.nchunks, T->npos[1] - 1, T->ncrd[1])
+        F1, F2, R, M, part.row, part.nz, part.aux, part.nchunks, T->npos[1] - 1, T->ncrd[1], T->dims[T->ord[0]], d1, d2)
         SP_DISPATCH_WIDTHS(T, {
             if (R % 4 == 0) SP_MTTKRP_FAST(4); else SP_MTTKRP_FAST(2);
         });
 #undef SP_MTTKRP_FAST
         SP_LAUNCH_CHECK();
         sp_count_launches(1);
+        SP_BOUNDS_RETURN(stream);
         return SP_OK;
     }
     SP_DISPATCH_WIDTHS(T, {
         k_mttkrp<P, I><<<blocks, kTThreads, 0, stream>>>(
             static_cast<const P*>(T->pos[1]), T->lt[0] == SP_COMPRESSED ? static_cast<const I*>(T->crd[0]) : nullptr,
             static_cast<const P*>(T->pos[2]), static_cast<const I*>(T->crd[1]), static_cast<const I*>(T->crd[2]),
-            T->val, F1, F2, R, M, part.row, part.nz, part.aux, part.nchunks, T->npos[1] - 1, T->ncrd[1]);
+            T->val, F1, F2, R, M, part.row, part.nz, part.aux, part.nchunks, T->npos[1] - 1, T->ncrd[1],
+            T->dims[T->ord[0]], d1, d2);
     });
     SP_LAUNCH_CHECK();
     sp_count_launches(1);
+    SP_BOUNDS_RETURN(stream);
     return SP_OK;
 }

@@ -75,44 +75,79 @@ struct LevelPlan {
 // ------------------------------------------------------------------ keys ---
 struct LevelCoords { const void* p[SP_MAX_RANK]; };   // coordinate array of the dimension stored at level l
 
-// idx_bits > 0: the entry index rides in the low idx_bits bits of the key itself (the sort then
-// moves 8 bytes per entry instead of 12) and no index array is written.
-template <typename CT>
-__global__ void k_build_keys(LevelCoords lc, int64_t n, LevelPlan p, uint64_t* keys, uint32_t* idx, int idx_bits,
-                             int* err) {
-    int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (e >= n) return;
-    uint64_t key = 0;
-    bool bad = false;
-#pragma unroll
-    for (int l = 0; l < SP_MAX_RANK; ++l) {
-        if (l < p.rank) {
-            CT c = static_cast<const CT*>(lc.p[l])[e];
-            if (c < 0 || (int64_t)c >= p.sz[l]) { bad = true; c = 0; }
-            key |= (uint64_t)c << p.shift[l];
-        }
-    }
-    if (bad) atomicOr(err, kErrRange);
-    if (idx_bits > 0) {
-        keys[e] = (key << idx_bits) | (uint64_t)e;
-    } else {
-        keys[e] = key;
-        idx[e] = (uint32_t)e;
-    }
-}
-
-// ------------------------------------------------------------ radix sort ---
-// Digits are up to kMaxDigitBits wide (512 bins): the 42-bit keys of a 16,384^3 tensor sort in five
-// passes (9, 9, 8, 8, 8 bits).  The kernels are instantiated per digit width so that the ranking
-// needs exactly that many ballots.
-#ifndef SP_SORT_MAX_BITS
-#define SP_SORT_MAX_BITS 9
-#endif
-constexpr int kMaxDigitBits = SP_SORT_MAX_BITS;
 constexpr int kSortThreads = 256;
 constexpr int kSortIpt = 16;
 constexpr int kSortTile = kSortThreads * kSortIpt;   // 4096
 constexpr int kSortWarps = kSortThreads / 32;
+constexpr int kMaxRadix = 256;
+
+// A block builds the keys of one sort tile and, while it has them in registers, the tile's digit
+// histogram for the first radix pass (digit = (key >> shift0) & mask0), so that pass needs no
+// counting sweep of its own.
+// idx_bits > 0: the entry index rides in the low idx_bits bits of the key itself (the sort then
+// moves 8 bytes per entry instead of 12) and no index array is written.
+template <typename CT>
+__global__ void __launch_bounds__(kSortThreads)
+k_build_keys(LevelCoords lc, int64_t n, LevelPlan p, uint64_t* keys, uint32_t* idx, int idx_bits, int* err,
+             int shift0, uint32_t mask0, uint32_t* __restrict__ tilehist, int64_t ntiles) {
+    __shared__ uint32_t hist[kSortWarps][kMaxRadix];
+    const int t = threadIdx.x, w = t >> 5;
+    for (int i = t; i < kSortWarps * kMaxRadix; i += kSortThreads) (&hist[0][0])[i] = 0;
+    __syncthreads();
+    const int64_t base = (int64_t)blockIdx.x * kSortTile;
+    CT c[kSortIpt / 2][SP_MAX_RANK];
+    bool bad = false;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+#pragma unroll
+        for (int i = 0; i < kSortIpt / 2; ++i) {       // the loads of eight entries first
+            const int64_t e = base + (int64_t)(half * (kSortIpt / 2) + i) * kSortThreads + t;
+#pragma unroll
+            for (int l = 0; l < SP_MAX_RANK; ++l)
+                if (l < p.rank) c[i][l] = e < n ? static_cast<const CT*>(lc.p[l])[e] : (CT)0;
+        }
+#pragma unroll
+        for (int i = 0; i < kSortIpt / 2; ++i) {
+            const int64_t e = base + (int64_t)(half * (kSortIpt / 2) + i) * kSortThreads + t;
+            if (e >= n) continue;
+            uint64_t key = 0;
+#pragma unroll
+            for (int l = 0; l < SP_MAX_RANK; ++l) {
+                if (l < p.rank) {
+                    CT v = c[i][l];
+                    if (v < 0 || (int64_t)v >= p.sz[l]) { bad = true; v = 0; }
+                    key |= (uint64_t)v << p.shift[l];
+                }
+            }
+            if (idx_bits > 0) {
+                key = (key << idx_bits) | (uint64_t)e;
+            } else {
+                idx[e] = (uint32_t)e;
+            }
+            keys[e] = key;
+            atomicAdd(&hist[w][(uint32_t)(key >> shift0) & mask0], 1u);
+        }
+    }
+    if (bad) atomicOr(err, kErrRange);
+    __syncthreads();
+    for (uint32_t d = t; d <= mask0; d += kSortThreads) {
+        uint32_t s = 0;
+#pragma unroll
+        for (int i = 0; i < kSortWarps; ++i) s += hist[i][d];
+        tilehist[(int64_t)d * ntiles + blockIdx.x] = s;
+    }
+}
+
+// ------------------------------------------------------------ radix sort ---
+// Digits are up to kMaxDigitBits wide: the 42-bit keys of a 16,384^3 tensor sort in six passes of
+// 7 bits.  (9-bit digits - five passes - were measured: each pass then costs 0.174 ms instead of
+// 0.145 ms on 20,000,000 entries and its histogram 0.039 ms instead of 0.034 ms, so nothing is won.)
+// The kernels are instantiated per digit width so that the ranking needs exactly that many ballots.
+#ifndef SP_SORT_MAX_BITS
+#define SP_SORT_MAX_BITS 8
+#endif
+constexpr int kMaxDigitBits = SP_SORT_MAX_BITS;
+static_assert((1 << kMaxDigitBits) <= kMaxRadix, "the key-building kernel's histogram holds kMaxRadix bins");
 
 __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
 #pragma unroll
@@ -141,6 +176,10 @@ __device__ __forceinline__ uint32_t block256_excl_scan(uint32_t v, uint32_t* sum
     return incl - v + pre;
 }
 
+// Tile histograms of one digit (passes after the first; the first pass's come from k_build_keys).
+// Counting them inside the previous pass's scatter, with global atomics where the keys land, was
+// measured: skewed digits pile onto few counters and the 20,000,000-entry scatter went from 0.145 ms
+// to 0.59 ms per pass.
 template <int BITS>
 __global__ void __launch_bounds__(kSortThreads)
 k_sort_upsweep(const uint64_t* __restrict__ keys, int64_t n, int shift, uint32_t* __restrict__ tilehist, int64_t ntiles) {
@@ -187,18 +226,38 @@ __device__ __forceinline__ uint32_t same_value_lanes(uint32_t d) {
     return peers;
 }
 
-// One block per digit: exclusive scan of that digit's tile counts, in place.
+// One block per digit: exclusive scan of that digit's tile counts, in place.  The counts are staged
+// in shared memory with coalesced loads; a thread then scans a contiguous run of them, and one block
+// scan joins the runs.
+constexpr int kScanChunk = 8192;
+
 __global__ void __launch_bounds__(256)
 k_sort_scan(uint32_t* tilehist, int64_t ntiles, uint32_t* digit_total) {
+    __shared__ uint32_t stage[kScanChunk];
     __shared__ uint32_t sums[8];
     uint32_t* row = tilehist + (int64_t)blockIdx.x * ntiles;
+    constexpr int kPer = kScanChunk / 256;
     uint32_t carry = 0;
-    for (int64_t base = 0; base < ntiles; base += 256) {
-        int64_t i = base + threadIdx.x;
-        uint32_t v = i < ntiles ? row[i] : 0u;
+    for (int64_t base = 0; base < ntiles; base += kScanChunk) {
+        const int cnt = (int)min((int64_t)kScanChunk, ntiles - base);
+        for (int i = threadIdx.x; i < cnt; i += 256) stage[i] = row[base + i];
+        __syncthreads();
+        uint32_t local = 0;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const int q = threadIdx.x * kPer + i;
+            if (q < cnt) local += stage[q];
+        }
         uint32_t tot;
-        uint32_t ex = block256_excl_scan(v, sums, &tot);
-        if (i < ntiles) row[i] = ex + carry;
+        uint32_t run = block256_excl_scan(local, sums, &tot) + carry;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const int q = threadIdx.x * kPer + i;
+            if (q < cnt) { const uint32_t v = stage[q]; stage[q] = run; run += v; }
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < cnt; i += 256) row[base + i] = stage[i];
+        __syncthreads();
         carry += tot;
     }
     if (threadIdx.x == 0) digit_total[blockIdx.x] = carry;
@@ -349,12 +408,16 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
     }
 }
 
-// One radix pass (histograms, per-digit scans, ranked scatter) for a digit of `bits` bits at `shift`.
+// One radix pass (tile histograms unless they exist already, per-digit scans, ranked scatter) for a
+// digit of BITS bits at `shift`.
 template <int BITS>
 sp_status sort_pass(const uint64_t* kin, const uint32_t* iin, uint64_t* kout, uint32_t* iout, int64_t n, int shift,
                     uint32_t* tilehist, int64_t stiles, uint32_t* digit_total, bool fused, int split_bits,
-                    cudaStream_t stream, PhaseTimer& timer) {
-    k_sort_upsweep<BITS><<<(unsigned)stiles, kSortThreads, 0, stream>>>(kin, n, shift, tilehist, stiles);
+                    bool have_hist, cudaStream_t stream, PhaseTimer& timer) {
+    if (!have_hist) {
+        k_sort_upsweep<BITS><<<(unsigned)stiles, kSortThreads, 0, stream>>>(kin, n, shift, tilehist, stiles);
+        sp_count_launches(1);
+    }
     timer.mark(kPhUpsweep);
     k_sort_scan<<<1 << BITS, 256, 0, stream>>>(tilehist, stiles, digit_total);
     timer.mark(kPhScan);
@@ -371,7 +434,7 @@ sp_status sort_pass(const uint64_t* kin, const uint32_t* iin, uint64_t* kout, ui
     }
     SP_LAUNCH_CHECK();
     timer.mark(kPhDownsweep);
-    sp_count_launches(3);
+    sp_count_launches(2);
     return SP_OK;
 }
 
@@ -777,37 +840,41 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         int idx_bits = 0;
         while (((int64_t)1 << idx_bits) < n) ++idx_bits;
         const bool fused = npasses > 0 && idx_bits > 0 && total_bits + idx_bits <= 64;
-        const unsigned kb = (unsigned)sp_ceil_div(n, 256);
+        // digit widths as even as possible, the wider ones first
+        int widths[16], shifts[16];
+        for (int ps = 0, kshift = 0; ps < npasses; ++ps) {
+            const int left = npasses - ps;
+            widths[ps] = (total_bits - kshift + left - 1) / left;
+            shifts[ps] = kshift + (fused ? idx_bits : 0);
+            kshift += widths[ps];
+        }
+        const int shift0 = npasses ? shifts[0] : 0;
+        const uint32_t mask0 = npasses ? (1u << widths[0]) - 1u : 0u;
         if (coo_coord_bits == 32)
-            k_build_keys<int32_t><<<kb, 256, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], fused ? idx_bits : 0, d_err);
+            k_build_keys<int32_t><<<(unsigned)stiles, kSortThreads, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], fused ? idx_bits : 0,
+                                                                              d_err, shift0, mask0, tilehist, stiles);
         else
-            k_build_keys<int64_t><<<kb, 256, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], fused ? idx_bits : 0, d_err);
+            k_build_keys<int64_t><<<(unsigned)stiles, kSortThreads, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], fused ? idx_bits : 0,
+                                                                              d_err, shift0, mask0, tilehist, stiles);
         SP_LAUNCH_CHECK();
         sp_count_launches(1);
         timer.mark(kPhKeys);
-        // digit widths as even as possible, the wider ones first (42 bits: 9, 9, 8, 8, 8)
-        int cur = 0, kshift = 0;
+        int cur = 0;
         for (int ps = 0; ps < npasses; ++ps) {
-            const int left = npasses - ps;
-            const int width = (total_bits - kshift + left - 1) / left;
-            const int shift = kshift + (fused ? idx_bits : 0);
-            const int split = (fused && ps == npasses - 1) ? idx_bits : -1;
+            const bool last = ps == npasses - 1;
+            const int split = (fused && last) ? idx_bits : -1;
             sp_status ps_st = SP_ERR_UNSUPPORTED;
 #define SP_SORT_PASS(B)                                                                                             \
     case B:                                                                                                         \
-        ps_st = sort_pass<B>(kbuf[cur], ibuf[cur], kbuf[cur ^ 1], ibuf[cur ^ 1], n, shift, tilehist, stiles,        \
-                             digit_total, fused, split, stream, timer);                                             \
+        ps_st = sort_pass<B>(kbuf[cur], ibuf[cur], kbuf[cur ^ 1], ibuf[cur ^ 1], n, shifts[ps], tilehist, stiles,    \
+                             digit_total, fused, split, ps == 0, stream, timer);                                     \
         break;
-            switch (width) {
+            switch (widths[ps]) {
                 SP_SORT_PASS(1) SP_SORT_PASS(2) SP_SORT_PASS(3) SP_SORT_PASS(4) SP_SORT_PASS(5)
                 SP_SORT_PASS(6) SP_SORT_PASS(7) SP_SORT_PASS(8)
-#if SP_SORT_MAX_BITS >= 9
-                SP_SORT_PASS(9)
-#endif
             }
 #undef SP_SORT_PASS
             if (ps_st != SP_OK) return ps_st;
-            kshift += width;
             cur ^= 1;
         }
         npasses_done = npasses;

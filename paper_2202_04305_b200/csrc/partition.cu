@@ -106,10 +106,7 @@ sp_status sp_get_segment_ids(sp_tensor* t, cudaStream_t stream, const uint32_t**
     std::lock_guard<std::mutex> lock(t->mu);
     const uint64_t key = (uint64_t)SP_PART_SEGIDS << 56;
     auto it = t->parts.find(key);
-    if (it != t->parts.end()) {
-        *out = reinterpret_cast<const uint32_t*>(it->second.aux);
-        return sp_partition_wait(it->second, stream);
-    }
+    if (it != t->parts.end()) { *out = reinterpret_cast<const uint32_t*>(it->second.aux); return SP_OK; }
     const int64_t nseg = t->npos[1] - 1, nnz = t->ncrd[1];
     sp_partition p;
     p.aux = static_cast<int64_t*>(sp_dev_alloc((size_t)(nnz ? nnz : 1) * sizeof(uint32_t), stream));
@@ -125,7 +122,7 @@ sp_status sp_get_segment_ids(sp_tensor* t, cudaStream_t stream, const uint32_t**
         if (cudaGetLastError() != cudaSuccess) { sp_dev_free(p.aux, stream); return SP_ERR_CUDA; }
         sp_count_launches(1);
     }
-    if (sp_partition_built(&p, stream) != SP_OK) { sp_dev_free(p.aux, stream); return SP_ERR_CUDA; }
+    if (sp_partition_built(stream) != SP_OK) { sp_dev_free(p.aux, stream); return SP_ERR_CUDA; }
     t->parts[key] = p;
     *out = seg;
     return SP_OK;
@@ -135,7 +132,7 @@ sp_status sp_get_merge_partition(sp_tensor* t, int64_t items, cudaStream_t strea
     std::lock_guard<std::mutex> lock(t->mu);
     const uint64_t key = ((uint64_t)SP_PART_MERGE_LAST << 56) | (uint64_t)items;
     auto it = t->parts.find(key);
-    if (it != t->parts.end()) { *out = it->second; return sp_partition_wait(it->second, stream); }
+    if (it != t->parts.end()) { *out = it->second; return SP_OK; }
     const int last = t->rank - 1;
     const int64_t nseg = t->npos[last] - 1;
     const int64_t nnz = t->ncrd[last];
@@ -155,7 +152,7 @@ sp_status sp_get_merge_partition(sp_tensor* t, int64_t items, cudaStream_t strea
                                                                  items, p.nchunks, p.row, p.nz);
     if (cudaGetLastError() != cudaSuccess) return drop(SP_ERR_CUDA);
     sp_count_launches(1);
-    if (sp_partition_built(&p, stream) != SP_OK) return drop(SP_ERR_CUDA);
+    if (sp_partition_built(stream) != SP_OK) return drop(SP_ERR_CUDA);
     t->parts[key] = p;
     *out = p;
     return SP_OK;
@@ -196,7 +193,7 @@ sp_status sp_widened(sp_tensor* t, cudaStream_t stream, sp_tensor** out) {
     std::lock_guard<std::mutex> lock(t->mu);
     if (t->wide) {
         *out = t->wide;
-        return sp_event_wait(t->wide_ready, t->wide_built_on, stream);
+        return SP_OK;
     }
     sp_tensor* w = new sp_tensor();
     w->rank = t->rank;
@@ -214,9 +211,7 @@ sp_status sp_widened(sp_tensor* t, cudaStream_t stream, sp_tensor** out) {
         if (st == SP_OK) st = widen_array(t->crd[l], t->ncrd[l], t->crdBits, stream, &w->crd[l]);
     }
     if (st != SP_OK) { sp_free(w); return st; }
-    if (cudaEventCreateWithFlags(&t->wide_ready, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventRecord(t->wide_ready, stream) != cudaSuccess) { sp_free(w); return SP_ERR_CUDA; }
-    t->wide_built_on = stream;
+    if (sp_partition_built(stream) != SP_OK) { sp_free(w); return SP_ERR_CUDA; }
     t->wide = w;
     *out = w;
     return SP_OK;
@@ -226,7 +221,7 @@ sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t per, cudaStream_t stream
     std::lock_guard<std::mutex> lock(t->mu);
     const uint64_t key = ((uint64_t)SP_PART_MTTKRP << 56) | (uint64_t)per;
     auto it = t->parts.find(key);
-    if (it != t->parts.end()) { *out = it->second; return sp_partition_wait(it->second, stream); }
+    if (it != t->parts.end()) { *out = it->second; return SP_OK; }
     const int64_t nnz = t->ncrd[2];
     const int64_t nfiber = t->ncrd[1];
     const int64_t nslice = t->npos[1] - 1;
@@ -249,7 +244,7 @@ sp_status sp_get_mttkrp_partition(sp_tensor* t, int64_t per, cudaStream_t stream
             p.nchunks, p.row, p.nz, p.aux);
     if (cudaGetLastError() != cudaSuccess) return drop(SP_ERR_CUDA);
     sp_count_launches(1);
-    if (sp_partition_built(&p, stream) != SP_OK) return drop(SP_ERR_CUDA);
+    if (sp_partition_built(stream) != SP_OK) return drop(SP_ERR_CUDA);
     t->parts[key] = p;
     *out = p;
     return SP_OK;

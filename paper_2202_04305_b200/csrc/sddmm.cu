@@ -46,7 +46,8 @@ __global__ void __launch_bounds__(kSThreads)
 k_sddmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ sval,
         const I* __restrict__ outer, const double* __restrict__ A, int64_t lda, const double* __restrict__ Bt,
         int64_t ldt, int64_t K, double* __restrict__ xv, const int64_t* __restrict__ prow,
-        const int64_t* __restrict__ pnz, int64_t nchunks) {
+        const int64_t* __restrict__ pnz, int64_t nchunks, int64_t na, int64_t nb) {
+    // na, nb: rows of A and of Bt (used by the bounds-checking debug build only)
     const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
     if (w >= nchunks) return;
     const int lane = threadIdx.x & 31;
@@ -66,7 +67,7 @@ k_sddmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __re
         const int64_t rend = row < i1 ? __shfl_sync(0xffffffffu, E, (int)(row - rbase)) : j1;
         const double* arow = nullptr;
         if (p < rend) {
-            arow = A + (outer ? (int64_t)outer[row] : row) * lda;
+            arow = A + SP_IDX(outer ? (int64_t)outer[row] : row, na) * lda;
             if (NCH > 0 && !a_ready) {
 #pragma unroll
                 for (int ch = 0; ch < NA; ++ch) {
@@ -89,7 +90,7 @@ k_sddmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __re
             }
             const int cnt = (int)min(rend - p, (int64_t)(32 - off));
             for (int t = 0; t < cnt; ++t) {
-                const int64_t j = (int64_t)__shfl_sync(0xffffffffu, c_l, off + t);
+                const int64_t j = SP_IDX(__shfl_sync(0xffffffffu, c_l, off + t), nb);
                 const double* brow = Bt + j * ldt;
                 double part = 0.0;
                 if (NCH > 0) {
@@ -139,7 +140,7 @@ template <typename I>
 __global__ void __launch_bounds__(256)
 k_sddmm_dense_inner(const I* __restrict__ outer, int64_t nouter, int64_t ninner, const double* __restrict__ sval,
                     const double* __restrict__ Out, int64_t out_row_stride, int64_t out_k_stride,
-                    const double* __restrict__ In, int64_t ldin, int64_t K, double* __restrict__ xv) {
+                    const double* __restrict__ In, int64_t ldin, int64_t K, double* __restrict__ xv, int64_t nouter_dim) {
     const int64_t c = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     for (int64_t q0 = (int64_t)blockIdx.y * kDQ; q0 < nouter; q0 += (int64_t)gridDim.y * kDQ) {
         const double* orow[kDQ];
@@ -147,7 +148,7 @@ k_sddmm_dense_inner(const I* __restrict__ outer, int64_t nouter, int64_t ninner,
 #pragma unroll
         for (int r = 0; r < kDQ; ++r) {
             const int64_t q = q0 + r < nouter ? q0 + r : nouter - 1;
-            orow[r] = Out + (outer ? (int64_t)outer[q] : q) * out_row_stride;
+            orow[r] = Out + SP_IDX(outer ? (int64_t)outer[q] : q, nouter_dim) * out_row_stride;
             acc[r] = 0.0;
         }
         if (c < ninner) {
@@ -193,10 +194,10 @@ sp_status sddmm_dense_inner(sp_tensor* S, const double* A, int64_t lda, const do
     dim3 grid((unsigned)sp_ceil_div(ninner, 256), (unsigned)std::min<int64_t>(sp_ceil_div(nouter, kDQ), 32768));
     if (S->crdBits == 32)
         k_sddmm_dense_inner<uint32_t><<<grid, 256, 0, stream>>>(dbl ? static_cast<const uint32_t*>(S->crd[0]) : nullptr, nouter,
-                                                               ninner, S->val, Out, out_row, out_k, In, ldin, K, x_vals);
+                                                               ninner, S->val, Out, out_row, out_k, In, ldin, K, x_vals, S->dims[S->ord[0]]);
     else
         k_sddmm_dense_inner<uint64_t><<<grid, 256, 0, stream>>>(dbl ? static_cast<const uint64_t*>(S->crd[0]) : nullptr, nouter,
-                                                               ninner, S->val, Out, out_row, out_k, In, ldin, K, x_vals);
+                                                               ninner, S->val, Out, out_row, out_k, In, ldin, K, x_vals, S->dims[S->ord[0]]);
     SP_LAUNCH_CHECK();
     sp_count_launches(1);
     return SP_OK;
@@ -251,7 +252,8 @@ extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const 
     }
 #define SP_SDDMM_LAUNCH(V, NCH)                                                                                     \
     k_sddmm<P, I, V, NCH><<<blocks, kSThreads, 0, stream>>>(pos, crd, S->val, outer, A, lda, Bt, ldt_k, K, x_vals,  \
-                                                            part.row, part.nz, part.nchunks)
+                                                            part.row, part.nz, part.nchunks, S->dims[S->ord[0]],   \
+                                                            S->dims[S->ord[1]])
     SP_DISPATCH_WIDTHS(S, {
         const P* pos = static_cast<const P*>(S->pos[1]);
         const I* crd = static_cast<const I*>(S->crd[1]);
@@ -268,5 +270,6 @@ extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const 
 #undef SP_SDDMM_LAUNCH
     SP_LAUNCH_CHECK();
     sp_count_launches(2);
+    SP_BOUNDS_RETURN(stream);
     return SP_OK;
 }

@@ -27,7 +27,8 @@ __global__ void __launch_bounds__(kVThreads)
 k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
        const I* __restrict__ outer, const double* __restrict__ x, double* __restrict__ y,
        const int64_t* __restrict__ prow, const int64_t* __restrict__ pnz, int64_t nseg,
-       double* __restrict__ carry_val, int64_t* __restrict__ carry_row) {
+       double* __restrict__ carry_val, int64_t* __restrict__ carry_row, int64_t m, int64_t n) {
+    // m, n: lengths of y and x (used by the bounds-checking debug build only)
     // a thread walks kVIpt consecutive products; one pad slot per kVIpt keeps those walks on distinct banks
     __shared__ int s_end[kVTile + 1];
     __shared__ double s_prod[kVTile + kVTile / kVIpt];
@@ -55,7 +56,7 @@ k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __res
         }
         if (!SCATTER) {
 #pragma unroll
-            for (int it = 0; it < kVIpt; ++it) xx[it] = __ldg(x + cc[it]);
+            for (int it = 0; it < kVIpt; ++it) xx[it] = __ldg(x + SP_IDX(cc[it], n));
         }
     }
     if (!SCATTER && nrows == 0) {
@@ -103,13 +104,13 @@ k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __res
     if (SCATTER) {
         // segment = a column of A; every entry adds val * x[col] into y[row]
         int64_t seg = i0 + ti;
-        double xc = seg < nseg ? x[outer ? (int64_t)outer[seg] : seg] : 0.0;
+        double xc = seg < nseg ? x[SP_IDX(outer ? (int64_t)outer[seg] : seg, n)] : 0.0;
         for (int s = d0; s < d1; ++s) {
             if (ti < nrows && s_end[ti] <= tj) {
                 ++ti; ++seg;
-                xc = seg < nseg ? x[outer ? (int64_t)outer[seg] : seg] : 0.0;
+                xc = seg < nseg ? x[SP_IDX(outer ? (int64_t)outer[seg] : seg, n)] : 0.0;
             } else {
-                atomicAdd(y + (int64_t)s_dst[SP_PAD(tj)], s_prod[SP_PAD(tj)] * xc);
+                atomicAdd(y + SP_IDX(s_dst[SP_PAD(tj)], m), s_prod[SP_PAD(tj)] * xc);
                 ++tj;
             }
         }
@@ -123,7 +124,7 @@ k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __res
             if (first_row < 0) { first_row = ti; first_val = run; }
             else {
                 const int64_t r = i0 + ti;
-                y[outer ? (int64_t)outer[r] : r] = run;
+                y[SP_IDX(outer ? (int64_t)outer[r] : r, m)] = run;
             }
             run = 0.0;
             ++ti;
@@ -156,7 +157,7 @@ k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __res
     (void)pf;
     if (first_row >= 0) {
         const int64_t r = i0 + first_row;
-        y[outer ? (int64_t)outer[r] : r] = first_val + in;
+        y[SP_IDX(outer ? (int64_t)outer[r] : r, m)] = first_val + in;
     }
     if (t == kVThreads - 1) {
         const double outv = (first_row >= 0) ? run : in + run;
@@ -168,14 +169,14 @@ k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __res
 
 template <typename I>
 __global__ void k_spmv_fixup(const double* __restrict__ carry_val, const int64_t* __restrict__ carry_row,
-                             int64_t ntiles, const I* __restrict__ outer, double* __restrict__ y) {
+                             int64_t ntiles, const I* __restrict__ outer, double* __restrict__ y, int64_t m) {
     int64_t w = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (w >= ntiles) return;
     const int64_t r = carry_row[w];
     if (r < 0 || (w > 0 && carry_row[w - 1] == r)) return;
     double s = 0.0;
     for (int64_t u = w; u < ntiles && carry_row[u] == r; ++u) s += carry_val[u];
-    y[outer ? (int64_t)outer[r] : r] += s;
+    y[SP_IDX(outer ? (int64_t)outer[r] : r, m)] += s;
 }
 
 // Row-major SpMV for matrices of short rows: G lanes per stored row, no staging, no carries.
@@ -185,7 +186,8 @@ __global__ void k_spmv_fixup(const double* __restrict__ carry_val, const int64_t
 template <typename P, typename I, int G>
 __global__ void __launch_bounds__(256)
 k_spmv_rows(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
-            const I* __restrict__ outer, const double* __restrict__ x, double* __restrict__ y, int64_t nseg) {
+            const I* __restrict__ outer, const double* __restrict__ x, double* __restrict__ y, int64_t nseg,
+            int64_t m, int64_t n, int64_t nnz) {
     constexpr int kU = 4;
     const int64_t q = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) / G;
     const int gl = threadIdx.x % G;
@@ -199,17 +201,17 @@ k_spmv_rows(const P* __restrict__ pos, const I* __restrict__ crd, const double* 
         for (int u = 0; u < kU; ++u) {
             const int64_t pp = p + u * G;
             const bool ok = pp < p1;
-            c[u] = ok ? crd[pp] : (I)0;
-            v[u] = ok ? val[pp] : 0.0;
+            c[u] = ok ? crd[SP_IDX(pp, nnz)] : (I)0;
+            v[u] = ok ? val[SP_IDX(pp, nnz)] : 0.0;
         }
 #pragma unroll
-        for (int u = 0; u < kU; ++u) xx[u] = (p + u * G < p1) ? __ldg(x + c[u]) : 0.0;
+        for (int u = 0; u < kU; ++u) xx[u] = (p + u * G < p1) ? __ldg(x + SP_IDX(c[u], n)) : 0.0;
 #pragma unroll
         for (int u = 0; u < kU; ++u) s = fma(v[u], xx[u], s);
     }
 #pragma unroll
     for (int o = G / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if (live && gl == 0) y[outer ? (int64_t)outer[q] : q] = s;
+    if (live && gl == 0) y[SP_IDX(outer ? (int64_t)outer[q] : q, m)] = s;
 }
 
 // ===================================================================== SpMM
@@ -246,7 +248,7 @@ k_spmm_gather(const P* __restrict__ pos, const I* __restrict__ crd, const double
               const I* __restrict__ outer, const double* __restrict__ B, int64_t N, int64_t ldb,
               double* __restrict__ C, int64_t ldc, const int64_t* __restrict__ prow,
               const int64_t* __restrict__ pnz, int64_t nchunks, int64_t nseg, double* __restrict__ carry,
-              int64_t* __restrict__ carry_row) {
+              int64_t* __restrict__ carry_row, int64_t m, int64_t n) {
     const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
     if (w >= nchunks) return;
     const int lane = threadIdx.x & 31;
@@ -272,7 +274,7 @@ k_spmm_gather(const P* __restrict__ pos, const I* __restrict__ crd, const double
         auto close_rows = [&](int64_t pe) {
             const int same = __popc(__ballot_sync(0xffffffffu, E == pe));
             for (int r = 0; r < same; ++r) {
-                if (on) st_vec<V>(C + (outer ? (int64_t)outer[row] : row) * ldc + col, acc);
+                if (on) st_vec<V>(C + SP_IDX(outer ? (int64_t)outer[row] : row, m) * ldc + col, acc);
 #pragma unroll
                 for (int q = 0; q < V; ++q) acc[q] = 0.0;
                 ++row;
@@ -313,7 +315,7 @@ k_spmm_gather(const P* __restrict__ pos, const I* __restrict__ crd, const double
 #pragma unroll
                 for (int u = 0; u < kG; ++u) {
                     if (g + u < cnt) {
-                        const int64_t k = (int64_t)__shfl_sync(0xffffffffu, c_l, g + u);
+                        const int64_t k = SP_IDX(__shfl_sync(0xffffffffu, c_l, g + u), n);
                         b[u] = ld_vec<V>(Bc + k * ldb);
                     }
                 }
@@ -345,7 +347,7 @@ template <typename I, int V>
 __global__ void __launch_bounds__(kMThreads)
 k_spmm_scatter(const uint32_t* __restrict__ seg, const I* __restrict__ crd, const double* __restrict__ val,
                int64_t nnz, const double* __restrict__ B, int64_t N, int64_t ldb, double* __restrict__ C,
-               int64_t ldc) {
+               int64_t ldc, int64_t m, int64_t n) {
     const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     const int64_t p0 = w * kScatPer;
@@ -366,14 +368,14 @@ k_spmm_scatter(const uint32_t* __restrict__ seg, const I* __restrict__ crd, cons
 #pragma unroll
                 for (int u = 0; u < kGather; ++u) {
                     if (g + u < cnt) {
-                        const int64_t k = (int64_t)__shfl_sync(0xffffffffu, k_l, g + u);
+                        const int64_t k = SP_IDX(__shfl_sync(0xffffffffu, k_l, g + u), n);
                         b[u] = ld_vec<V>(Bc + k * ldb);
                     }
                 }
 #pragma unroll
                 for (int u = 0; u < kGather; ++u) {
                     if (g + u < cnt) {
-                        const int64_t i = (int64_t)__shfl_sync(0xffffffffu, i_l, g + u);
+                        const int64_t i = SP_IDX(__shfl_sync(0xffffffffu, i_l, g + u), m);
                         const double vv = __shfl_sync(0xffffffffu, v_l, g + u);
                         if (on) {
 #pragma unroll
@@ -389,7 +391,7 @@ k_spmm_scatter(const uint32_t* __restrict__ seg, const I* __restrict__ crd, cons
 template <typename I>
 __global__ void k_spmm_fixup(const double* __restrict__ carry, const int64_t* __restrict__ carry_row,
                              int64_t nchunks, const I* __restrict__ outer, int64_t N, double* __restrict__ C,
-                             int64_t ldc) {
+                             int64_t ldc, int64_t m) {
     const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
     if (w >= nchunks) return;
     const int lane = threadIdx.x & 31;
@@ -397,7 +399,7 @@ __global__ void k_spmm_fixup(const double* __restrict__ carry, const int64_t* __
     if (r < 0 || (w > 0 && carry_row[w - 1] == r)) return;
     int64_t end = w + 1;
     while (end < nchunks && carry_row[end] == r) ++end;
-    double* crow = C + (outer ? (int64_t)outer[r] : r) * ldc;
+    double* crow = C + SP_IDX(outer ? (int64_t)outer[r] : r, m) * ldc;
     for (int64_t col = lane; col < N; col += 32) {
         double s = 0.0;
         for (int64_t u = w; u < end; ++u) s += carry[u * N + col];
@@ -447,13 +449,14 @@ extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* str
                 const P* pos = static_cast<const P*>(A->pos[1]);
                 const I* crd = static_cast<const I*>(A->crd[1]);
                 const I* outer = dbl ? static_cast<const I*>(A->crd[0]) : nullptr;
-                if (G == 4) k_spmv_rows<P, I, 4><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg);
-                else if (G == 8) k_spmv_rows<P, I, 8><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg);
-                else if (G == 16) k_spmv_rows<P, I, 16><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg);
-                else k_spmv_rows<P, I, 32><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg);
+                if (G == 4) k_spmv_rows<P, I, 4><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg, m, A->dims[1], A->ncrd[1]);
+                else if (G == 8) k_spmv_rows<P, I, 8><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg, m, A->dims[1], A->ncrd[1]);
+                else if (G == 16) k_spmv_rows<P, I, 16><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg, m, A->dims[1], A->ncrd[1]);
+                else k_spmv_rows<P, I, 32><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg, m, A->dims[1], A->ncrd[1]);
             });
             SP_LAUNCH_CHECK();
             sp_count_launches(1);
+            SP_BOUNDS_RETURN(stream);
             return SP_OK;
         }
     }
@@ -471,16 +474,17 @@ extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* str
         const I* outer = dbl ? static_cast<const I*>(A->crd[0]) : nullptr;
         if (rowmajor) {
             k_spmv<P, I, false><<<(unsigned)part.nchunks, kVThreads, 0, stream>>>(pos, crd, A->val, outer, x, y, part.row,
-                                                                                  part.nz, nseg, cval, crow);
-            k_spmv_fixup<I><<<(unsigned)sp_ceil_div(part.nchunks, 256), 256, 0, stream>>>(cval, crow, part.nchunks, outer, y);
+                                                                                  part.nz, nseg, cval, crow, m, A->dims[1]);
+            k_spmv_fixup<I><<<(unsigned)sp_ceil_div(part.nchunks, 256), 256, 0, stream>>>(cval, crow, part.nchunks, outer, y, m);
             sp_count_launches(2);
         } else {
             k_spmv<P, I, true><<<(unsigned)part.nchunks, kVThreads, 0, stream>>>(pos, crd, A->val, outer, x, y, part.row,
-                                                                                 part.nz, nseg, cval, crow);
+                                                                                 part.nz, nseg, cval, crow, m, A->dims[1]);
             sp_count_launches(1);
         }
     });
     SP_LAUNCH_CHECK();
+    SP_BOUNDS_RETURN(stream);
     return SP_OK;
 }
 
@@ -540,24 +544,25 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
         if (rowmajor) {
             if (vec2)
                 k_spmm_gather<P, I, 2><<<blocks, kMThreads, 0, stream>>>(pos, crd, A->val, outer, B, N, ldb, C, ldc, part.row,
-                                                                         part.nz, part.nchunks, nseg, carry, crow);
+                                                                         part.nz, part.nchunks, nseg, carry, crow, m, A->dims[1]);
             else
                 k_spmm_gather<P, I, 1><<<blocks, kMThreads, 0, stream>>>(pos, crd, A->val, outer, B, N, ldb, C, ldc, part.row,
-                                                                         part.nz, part.nchunks, nseg, carry, crow);
-            k_spmm_fixup<I><<<blocks, kMThreads, 0, stream>>>(carry, crow, part.nchunks, outer, N, C, ldc);
+                                                                         part.nz, part.nchunks, nseg, carry, crow, m, A->dims[1]);
+            k_spmm_fixup<I><<<blocks, kMThreads, 0, stream>>>(carry, crow, part.nchunks, outer, N, C, ldc, m);
             sp_count_launches(2);
         } else {
             (void)pos;
             const int64_t nnz = A->ncrd[1];
             const unsigned sblocks = (unsigned)sp_ceil_div(sp_ceil_div(nnz, kScatPer) * 32, kMThreads);
             if (nnz > 0) {
-                if (vec2) k_spmm_scatter<I, 2><<<sblocks, kMThreads, 0, stream>>>(segs, crd, A->val, nnz, B, N, ldb, C, ldc);
-                else k_spmm_scatter<I, 1><<<sblocks, kMThreads, 0, stream>>>(segs, crd, A->val, nnz, B, N, ldb, C, ldc);
+                if (vec2) k_spmm_scatter<I, 2><<<sblocks, kMThreads, 0, stream>>>(segs, crd, A->val, nnz, B, N, ldb, C, ldc, m, A->dims[1]);
+                else k_spmm_scatter<I, 1><<<sblocks, kMThreads, 0, stream>>>(segs, crd, A->val, nnz, B, N, ldb, C, ldc, m, A->dims[1]);
                 sp_count_launches(1);
             }
         }
     });
     SP_LAUNCH_CHECK();
+    SP_BOUNDS_RETURN(stream);
     return SP_OK;
 }
 
@@ -648,13 +653,13 @@ extern "C" sp_status sp_spmv_static(const sp_tensor* A, const double* x, double*
                                                                                           sc->nz);
         if (rowmajor) {
             k_spmv<P, I, false><<<(unsigned)ntiles, kVThreads, 0, stream>>>(pos, crd, A->val, outer, x, y, sc->row, sc->nz,
-                                                                            nseg, sc->carry_val, sc->carry_row);
+                                                                            nseg, sc->carry_val, sc->carry_row, A->dims[0], A->dims[1]);
             k_spmv_fixup<I><<<(unsigned)sp_ceil_div(ntiles, 256), 256, 0, stream>>>(sc->carry_val, sc->carry_row, ntiles,
-                                                                                    outer, y);
+                                                                                    outer, y, A->dims[0]);
             sp_count_launches(3);
         } else {
             k_spmv<P, I, true><<<(unsigned)ntiles, kVThreads, 0, stream>>>(pos, crd, A->val, outer, x, y, sc->row, sc->nz,
-                                                                           nseg, sc->carry_val, sc->carry_row);
+                                                                           nseg, sc->carry_val, sc->carry_row, A->dims[0], A->dims[1]);
             sp_count_launches(2);
         }
     });

@@ -40,9 +40,9 @@ def test_static_matches_spmv_two_calls_in_a_row(oracle, enc, widths):
             got, ref = _both(A, dev(x))
             exact, bound = oracle.spmv(coo.dims[0], coo.coords[0], coo.coords[1], coo.vals, x)
             assert_close(got, exact, bound, f"static {enc} call {rep}")
+            # sp_spmv may take another route over the same storage (a lane group per row for short
+            # rows), so the two agree to rounding, not bit for bit
             assert np.all(np.abs(got - ref) <= 2 * TOL * bound)
-            if od == (0, 1):                                # no atomics: identical arithmetic, identical bits
-                assert np.array_equal(got, ref)
 
 
 def test_static_never_calls_the_allocator_and_rejects_oversize():
@@ -75,7 +75,7 @@ def test_static_never_calls_the_allocator_and_rejects_oversize():
         assert len(calls) > 0
     finally:
         assert b._lib.sp_set_allocator(b._alloc_cb, b._free_cb, None) == 0
-    assert np.array_equal(y.cpu().numpy(), b.sp_spmv(A, x).cpu().numpy())
+    assert np.allclose(y.cpu().numpy(), b.sp_spmv(A, x).cpu().numpy(), rtol=0, atol=1e-12)   # same product, maybe another route
 
     # more (row ends + entries) than the fixed scratch can describe: refused, nothing launched
     rows = b.SPMV_STATIC_MAX_ITEMS + 5
