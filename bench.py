@@ -534,6 +534,86 @@ def run_reference(args, wl, model, total_flops, cfg):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------- one call on its own (for profilers)
+def run_only_call(name: str, reps: int, seed: int = 0):
+    """One call of the step at full size, `reps` times after a warm-up call, bracketed by
+    cudaProfilerStart/Stop: builds only the inputs that call needs, so that a profiler capture
+    (`ncu --profile-from-start off -k regex:... -c N python bench.py --only-call NAME`) holds little
+    memory and runs few launches.  `probe_<bytes>B_<table MB>MB` runs the row-gather probe instead."""
+    import torch
+    import paper_2202_04305_b200.binding as sp
+    dev = lambda a: torch.as_tensor(np.ascontiguousarray(a), device="cuda")
+    i32 = lambda c: [dev(x.astype(np.int32)) for x in c.coords]
+    f64 = lambda *sh: torch.empty(sh, dtype=torch.float64, device="cuda")
+    if name.startswith("probe_"):
+        row_bytes, table_mb = (int(x.rstrip("BM")) for x in name[len("probe_"):].split("_"))
+        probes = Probes()
+        elems = row_bytes // 8
+        rows = max(1, (table_mb << 20) // row_bytes) if table_mb > 0 else max(1, L1_TABLE_BYTES // row_bytes)
+        table = torch.rand(rows, elems, dtype=torch.float64, device="cuda") if elems > 1 else torch.rand(rows, dtype=torch.float64, device="cuda")
+        blocks = torch.cuda.get_device_properties(0).multi_processor_count * 8
+        ids = torch.randint(0, rows, (blocks * 8 * 256 * 64,), dtype=torch.int32, device="cuda")
+        fn = lambda: probes.gather_rows(table, ids, blocks)
+    elif name in ("pack_csc", "pack_dcsr", "spmm_csc", "spmm_dcsr", "spmv_dcsr"):
+        c = I.config3(seed)
+        coords, vals = i32(c), dev(c.vals)
+        lt, od = ((0, 1), (1, 0)) if name.endswith("csc") else ((1, 1), None)
+        if name.startswith("pack"):
+            fn = lambda: sp.sp_pack(c.dims, coords, vals, lt, od).free()
+        else:
+            A = sp.sp_pack(c.dims, coords, vals, lt, od)
+            if name.startswith("spmm"):
+                B, C = dev(I.dense_operand(seed, 31, c.dims[1], 32)), f64(c.dims[0], 32)
+                fn = lambda: sp.sp_spmm(A, B, C)
+            else:
+                x, y = dev(I.uniform_pm1(seed, 32, c.dims[1])), f64(c.dims[0])
+                fn = lambda: sp.sp_spmv(A, x, y)
+    elif name in ("spmm_csr", "spmv_csr_powerlaw"):
+        c = I.config2(seed)
+        A = sp.sp_pack(c.dims, i32(c), dev(c.vals), (0, 1))
+        if name == "spmm_csr":
+            B, C = dev(I.dense_operand(seed, 33, c.dims[1], 64)), f64(c.dims[0], 64)
+            fn = lambda: sp.sp_spmm(A, B, C)
+        else:
+            x, y = dev(I.uniform_pm1(seed, 32, c.dims[1])), f64(c.dims[0])
+            fn = lambda: sp.sp_spmv(A, x, y)
+    elif name in ("spmv_csr", "spmv_cdr", "next_spmm_cdr"):
+        c = I.config1b(seed)
+        A = sp.sp_pack(c.dims, i32(c), dev(c.vals), (0, 1) if name == "spmv_csr" else (1, 0))
+        if name == "next_spmm_cdr":
+            B, C = torch.rand(c.dims[1], 32, dtype=torch.float64, device="cuda"), f64(c.dims[0], 32)
+            fn = lambda: sp.sp_spmm(A, B, C)
+        else:
+            x, y = dev(I.uniform_pm1(seed, 34, c.dims[1])), f64(c.dims[0])
+            fn = lambda: sp.sp_spmv(A, x, y)
+    elif name == "sddmm_csr":
+        c = I.config4(seed)
+        S = sp.sp_pack(c.dims, i32(c), dev(c.vals), (0, 1))
+        A4, B4, xv = dev(I.dense_operand(seed, 35, c.dims[0], 128)), dev(I.dense_operand(seed, 36, 128, c.dims[1])), f64(S.nval)
+        fn = lambda: sp.sp_sddmm(S, A4, B4, xv)
+    elif name in ("pack_csf", "mttkrp_csf"):
+        c = I.config5(seed)
+        coords, vals = i32(c), dev(c.vals)
+        if name == "pack_csf":
+            fn = lambda: sp.sp_pack(c.dims, coords, vals, (1, 1, 1)).free()
+        else:
+            T = sp.sp_pack(c.dims, coords, vals, (1, 1, 1))
+            Bf, Cf, M = dev(I.dense_operand(seed, 37, c.dims[1], 32)), dev(I.dense_operand(seed, 38, c.dims[2], 32)), f64(c.dims[0], 32)
+            fn = lambda: sp.sp_mttkrp(T, Bf, Cf, M)
+    else:
+        raise SystemExit(f"unknown call {name}")
+    fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.profiler.start()
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record(); torch.cuda.synchronize()
+    torch.cuda.profiler.stop()
+    print(json.dumps({"only_call": name, "reps": reps, "ms_per_call_warm_l2": round(a.elapsed_time(b) / reps, 4)}))
+
+
 # --------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -544,11 +624,17 @@ def main():
     ap.add_argument("--small", action="store_true", help="reduced sizes (development runs; not a valid benchmark)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel-reps", type=int, default=20)
+    ap.add_argument("--only-call", default=None,
+                    help="run one named call of the step (or probe_<row bytes>B_<table MB>MB) on its own, for a profiler capture")
+    ap.add_argument("--reps", type=int, default=3, help="repetitions for --only-call")
     ap.add_argument("--only-step", action="store_true",
                     help="run only the timed steps, bracketed by cudaProfilerStart/Stop (for `ncu --profile-from-start off`)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank, local_rank, world = dist_env()
+    if args.only_call:
+        run_only_call(args.only_call, args.reps)
+        return
 
     wl = make_workload(args.small, seed=rank if args.impl == "ours" else 0)
     model = work_model(wl)
