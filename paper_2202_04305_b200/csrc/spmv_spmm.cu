@@ -22,8 +22,11 @@ constexpr int kVThreads = 256;
 constexpr int kVIpt = 8;
 constexpr int kVTile = kVThreads * kVIpt;   // merge items per CTA
 
+#ifndef SP_LB_SPMV
+#define SP_LB_SPMV 1
+#endif
 template <typename P, typename I, bool SCATTER>
-__global__ void __launch_bounds__(kVThreads)
+__global__ void __launch_bounds__(kVThreads, SP_LB_SPMV)
 k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
        const I* __restrict__ outer, const double* __restrict__ x, double* __restrict__ y,
        const int64_t* __restrict__ prow, const int64_t* __restrict__ pnz, int64_t nseg,
@@ -182,7 +185,9 @@ __global__ void k_spmv_fixup(const double* __restrict__ carry_val, const int64_t
 // Row-major SpMV for matrices of short rows: G lanes per stored row, no staging, no carries.
 // Every lane issues its (up to four) coordinate and value loads, then the gathered x entries,
 // before the first multiply-add; the row's sum is folded over the group's lanes and written once.
-// Rows without entries (CSR) are written as zeros here; rows that DCSR elides were zeroed before.
+// Rows without entries (CSR) are written as zeros here; when level 0 is compressed the group of
+// stored row q also writes the zeros of the rows that storage elides between stored rows q - 1 and q
+// (the last group those after its row too), so y needs no clearing pass.
 template <typename P, typename I, int G>
 __global__ void __launch_bounds__(256)
 k_spmv_rows(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
@@ -211,7 +216,15 @@ k_spmv_rows(const P* __restrict__ pos, const I* __restrict__ crd, const double* 
     }
 #pragma unroll
     for (int o = G / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if (live && gl == 0) y[SP_IDX(outer ? (int64_t)outer[q] : q, m)] = s;
+    if (!live) return;
+    const int64_t row = SP_IDX(outer ? (int64_t)outer[q] : q, m);
+    if (gl == 0) y[row] = s;
+    if (outer) {
+        const int64_t gap0 = q > 0 ? SP_IDX(outer[q - 1], m) + 1 : 0;
+        for (int64_t r = gap0 + gl; r < row; r += G) y[r] = 0.0;
+        if (q == nseg - 1)
+            for (int64_t r = row + 1 + gl; r < m; r += G) y[r] = 0.0;
+    }
 }
 
 // ===================================================================== SpMM
@@ -341,9 +354,14 @@ k_spmm_gather(const P* __restrict__ pos, const I* __restrict__ crd, const double
 // carried between rows.  The lanes of a group read whole 16 * L-byte runs of a B row per load
 // instruction (lane gl holds column pairs gl, gl + L, ...), and a lane has the loads of kU entries
 // (16 loads of 16 bytes) in flight before the first multiply-add - the access pattern that fetches
-// random rows fastest on this GPU.  Rows without entries are written as zeros.
+// random rows fastest on this GPU.  Rows without entries are written as zeros; when level 0 is
+// compressed the group of stored row q also writes the zeros of the rows that storage elides between
+// stored rows q - 1 and q (the last group those after its row too), so that C needs no clearing pass.
+#ifndef SP_SPMM_ROWS_THREADS
+#define SP_SPMM_ROWS_THREADS 256
+#endif
 template <typename P, typename I, int L, int V>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(SP_SPMM_ROWS_THREADS)
 k_spmm_rows(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
             const I* __restrict__ outer, const double* __restrict__ B, int64_t ldb, double* __restrict__ C,
             int64_t ldc, int64_t nseg, int64_t m, int64_t n) {
@@ -356,23 +374,33 @@ k_spmm_rows(const P* __restrict__ pos, const I* __restrict__ crd, const double* 
     double acc[V];
 #pragma unroll
     for (int j = 0; j < V; ++j) acc[j] = 0.0;
+    // coordinates and values are fetched one turn ahead, so that a turn's B rows can be requested at once
+    I kn[kU];
+    double vn[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {                  // the group's lanes read the same word: one transaction
+        const bool ok = p0 + u < p1;
+        kn[u] = ok ? crd[p0 + u] : (I)0;
+        vn[u] = ok ? val[p0 + u] : 0.0;
+    }
     for (int64_t p = p0; p < p1; p += kU) {
         int64_t k[kU];
         double v[kU];
         double2 b[kU][V / 2];
 #pragma unroll
-        for (int u = 0; u < kU; ++u) {              // the group's lanes read the same word: one transaction
-            const bool ok = p + u < p1;
-            k[u] = ok ? (int64_t)SP_IDX(crd[p + u], n) : 0;
-            v[u] = ok ? val[p + u] : 0.0;
-        }
+        for (int u = 0; u < kU; ++u) { k[u] = (int64_t)SP_IDX(kn[u], n); v[u] = vn[u]; }
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
 #pragma unroll
             for (int j = 0; j < V / 2; ++j)
                 b[u][j] = (p + u < p1) ? *reinterpret_cast<const double2*>(Bl + k[u] * ldb + j * 2 * L) : make_double2(0.0, 0.0);
         }
-        asm volatile("" ::: "memory");              // every load above is issued before the first multiply-add below
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const bool ok = p + kU + u < p1;
+            kn[u] = ok ? crd[p + kU + u] : (I)0;
+            vn[u] = ok ? val[p + kU + u] : 0.0;
+        }
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
 #pragma unroll
@@ -382,9 +410,20 @@ k_spmm_rows(const P* __restrict__ pos, const I* __restrict__ crd, const double* 
             }
         }
     }
-    double* crow = C + SP_IDX(outer ? (int64_t)outer[q] : q, m) * ldc + 2 * gl;
+    const int64_t row = SP_IDX(outer ? (int64_t)outer[q] : q, m);
+    double* crow = C + row * ldc + 2 * gl;
 #pragma unroll
     for (int j = 0; j < V / 2; ++j) *reinterpret_cast<double2*>(crow + j * 2 * L) = make_double2(acc[2 * j], acc[2 * j + 1]);
+    if (outer) {
+        const int64_t gap0 = q > 0 ? SP_IDX(outer[q - 1], m) + 1 : 0;
+        for (int64_t r = gap0; r < row; ++r)
+#pragma unroll
+            for (int j = 0; j < V / 2; ++j) *reinterpret_cast<double2*>(C + r * ldc + 2 * gl + j * 2 * L) = make_double2(0.0, 0.0);
+        if (q == nseg - 1)
+            for (int64_t r = row + 1; r < m; ++r)
+#pragma unroll
+                for (int j = 0; j < V / 2; ++j) *reinterpret_cast<double2*>(C + r * ldc + 2 * gl + j * 2 * L) = make_double2(0.0, 0.0);
+    }
 }
 
 // Column-major SpMM (CSC, DCSC): C[i,:] += A[i,k] * B[k,:] for every stored entry, as a flat loop
@@ -482,9 +521,11 @@ extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* str
     const bool rowmajor = A->ord[0] == 0;
     const bool dbl = A->lt[0] == SP_COMPRESSED;
     const int64_t m = A->dims[0];
-    if (!rowmajor || dbl) SP_CUDA(cudaMemsetAsync(y, 0, (size_t)m * sizeof(double), stream));
     const int64_t nseg = A->npos[1] - 1;
-    if (nseg <= 0) return SP_OK;
+    if (nseg <= 0 || A->ncrd[1] == 0 || (dbl && A->ncrd[0] == 0)) {
+        SP_CUDA(cudaMemsetAsync(y, 0, (size_t)m * sizeof(double), stream));
+        return SP_OK;
+    }
     // Short rows (mean <= 256 entries, none longer than 4096): a lane group per row, one launch.
     // Anything skewed or long goes through the merge path below, whose cost does not depend on the
     // row lengths.
@@ -515,6 +556,7 @@ extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* str
             return SP_OK;
         }
     }
+    if (!rowmajor || dbl) SP_CUDA(cudaMemsetAsync(y, 0, (size_t)m * sizeof(double), stream));
     sp_partition part;
     sp_status st = sp_get_merge_partition(A, kVTile, stream, &part);
     if (st != SP_OK) return st;
@@ -562,12 +604,13 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
     const bool rowmajor = A->ord[0] == 0;
     const bool dbl = A->lt[0] == SP_COMPRESSED;
     const int64_t m = A->dims[0];
-    if (!rowmajor || dbl) {
+    auto clear_C = [&]() -> sp_status {
         if (ldc == N) SP_CUDA(cudaMemsetAsync(C, 0, (size_t)m * N * sizeof(double), stream));
         else SP_CUDA(cudaMemset2DAsync(C, (size_t)ldc * sizeof(double), 0, (size_t)N * sizeof(double), (size_t)m, stream));
-    }
+        return SP_OK;
+    };
     const int64_t nseg = A->npos[1] - 1;
-    if (nseg <= 0) return SP_OK;
+    if (nseg <= 0 || A->ncrd[1] == 0 || (dbl && A->ncrd[0] == 0)) return clear_C();
     // column-major storage runs as a flat loop over entries with their column ids expanded once
     // (32-bit ids: a column-major matrix with 2^32 or more columns is refused)
     if (!rowmajor && A->dims[1] >= ((int64_t)1 << 32)) return SP_ERR_UNSUPPORTED;
@@ -575,8 +618,9 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
     sp_status st = SP_OK;
     // Rows of similar, moderate length (the longest at most four mean lengths + 32, and no more than
     // 4096 entries), N = 16, 32, 64 or 128 and 16-byte aligned operands: a lane group per row.
-    // Skewed matrices stay on the merge path, whose pieces cost the same whatever the row lengths
-    // (power-law rows of mean 16, up to 435 long, N = 64: 0.091 ms there against 0.23 ms here).
+    // Skewed matrices stay on the merge path, whose pieces cost the same whatever the row lengths.
+    // Measured on power-law rows (mean 16, up to 435 long, N = 64): merge path 0.091 ms, a lane group per
+    // row 0.23 ms, lane groups for the rows up to 96 long plus a block for each longer one 0.16 ms.
     if (rowmajor && (N == 16 || N == 32 || N == 64 || N == 128) && ldb % 2 == 0 && ldc % 2 == 0 &&
         reinterpret_cast<uintptr_t>(B) % 16 == 0 && reinterpret_cast<uintptr_t>(C) % 16 == 0) {
         int64_t max_seg = 0;
@@ -584,9 +628,9 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
         if (st != SP_OK) return st;
         const int64_t mean = A->ncrd[1] / nseg;
         if (max_seg <= 4096 && max_seg <= 4 * mean + 32) {
-#define SP_SPMM_ROWS(L, V)                                                                                    \
-    k_spmm_rows<P, I, L, V><<<(unsigned)sp_ceil_div(nseg * L, 256), 256, 0, stream>>>(pos, crd, A->val, outer, B, ldb, C, \
-                                                                                      ldc, nseg, m, A->dims[1])
+#define SP_SPMM_ROWS(L, V)                                                                                              \
+    k_spmm_rows<P, I, L, V><<<(unsigned)sp_ceil_div(nseg * L, SP_SPMM_ROWS_THREADS), SP_SPMM_ROWS_THREADS, 0, stream>>>( \
+        pos, crd, A->val, outer, B, ldb, C, ldc, nseg, m, A->dims[1])
             SP_DISPATCH_WIDTHS(A, {
                 const P* pos = static_cast<const P*>(A->pos[1]);
                 const I* crd = static_cast<const I*>(A->crd[1]);
@@ -602,6 +646,10 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
             SP_BOUNDS_RETURN(stream);
             return SP_OK;
         }
+    }
+    if (!rowmajor || dbl) {            // rows that storage elides, and scatter targets, start from zero
+        st = clear_C();
+        if (st != SP_OK) return st;
     }
     sp_partition part;
     sp_workspace ws(stream);

@@ -107,6 +107,38 @@ def test_spmm_strided_operands_and_wide_indices(oracle):
             assert torch.all(Cbig[:, 48:] == 7.0)
 
 
+@pytest.mark.parametrize("N", [16, 32, 64, 128])
+@pytest.mark.parametrize("lt", [(0, 1), (1, 1)])
+def test_spmm_lane_group_per_row(oracle, N, lt):
+    """Rows of even, moderate length take the lane-group kernel (N = 16, 32, 64, 128): stored rows, rows
+    without entries (written as zeros, including those a compressed level 0 elides before the first,
+    between, and after the last stored row), a strided C whose other columns must stay untouched, and
+    every index width."""
+    import torch
+    m, n = 900, 700
+    rows = np.setdiff1d(np.arange(5, m - 9), np.arange(100, 140))       # rows 0-4, 100-139 and the last 9 hold nothing
+    r = np.repeat(rows, 12)
+    c = (I.randint(21, 1, r.size, n // 12) + np.tile(np.arange(12) * (n // 12), rows.size)).astype(np.int64)   # distinct per row
+    v = I.uniform_pm1(21, 2, r.size)
+    perm = I.affine_scramble(r.size, 3)
+    coo = I.Coo((m, n), [r[perm], c[perm]], v[perm])
+    B = I.dense_operand(21, 3, n, N)
+    ref, bd = oracle.spmm(m, coo.coords[0], coo.coords[1], coo.vals, B)
+    for pb, cb, cbits in [(32, 32, 32), (64, 64, 64), (32, 64, 32), (64, 32, 64)]:
+        coords, vals = to_dev(coo, cbits)
+        A = sp().sp_pack(coo.dims, coords, vals, lt, None, pb, cb)
+        Bbig = torch.zeros((n, N + 2), dtype=torch.float64, device="cuda")
+        Bbig[:, :N] = dev(B)
+        Cbig = torch.full((m, N + 4), 7.0, dtype=torch.float64, device="cuda")
+        sp().sp_spmm(A, Bbig[:, :N], Cbig[:, :N])
+        assert_close(Cbig[:, :N].cpu().numpy(), ref, bd, f"rows {lt} N={N}")
+        assert torch.all(Cbig[:, N:] == 7.0)
+        x = I.uniform_pm1(21, 4, n)
+        yref, yb = oracle.spmv(m, coo.coords[0], coo.coords[1], coo.vals, x)
+        y = torch.full((m,), 7.0, dtype=torch.float64, device="cuda")
+        assert_close(sp().sp_spmv(A, dev(x), y).cpu().numpy(), yref, yb, f"spmv rows {lt}")
+
+
 def test_results_do_not_depend_on_encoding(oracle):
     # Section 5.2: the result is independent of the sparsity annotation, up to reassociation.
     coo = I.uniform_matrix(500, 400, 9000, seed=21)
