@@ -192,8 +192,11 @@ __device__ __forceinline__ void ld_cols(const double* p, const int* coff, double
     }
 }
 
+#ifndef SP_LB_MTTKRP
+#define SP_LB_MTTKRP 2
+#endif
 template <typename P, typename I, int S>
-__global__ void __launch_bounds__(kTThreads)
+__global__ void __launch_bounds__(kTThreads, SP_LB_MTTKRP)
 k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* __restrict__ pos2,
               const I* __restrict__ crd1, const I* __restrict__ crd2, const double* __restrict__ val,
               const double* __restrict__ F1, const double* __restrict__ F2, int64_t R, double* __restrict__ M,

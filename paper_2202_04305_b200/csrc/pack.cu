@@ -75,8 +75,17 @@ struct LevelPlan {
 // ------------------------------------------------------------------ keys ---
 struct LevelCoords { const void* p[SP_MAX_RANK]; };   // coordinate array of the dimension stored at level l
 
-constexpr int kSortThreads = 256;
-constexpr int kSortIpt = 16;
+#ifndef SP_SORT_THREADS
+#define SP_SORT_THREADS 256
+#endif
+#ifndef SP_SORT_IPT
+#define SP_SORT_IPT 16
+#endif
+#ifndef SP_SORT_MIN_BLOCKS
+#define SP_SORT_MIN_BLOCKS 3
+#endif
+constexpr int kSortThreads = SP_SORT_THREADS;
+constexpr int kSortIpt = SP_SORT_IPT;
 constexpr int kSortTile = kSortThreads * kSortIpt;   // 4096
 constexpr int kSortWarps = kSortThreads / 32;
 constexpr int kMaxRadix = 256;
@@ -158,15 +167,16 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
     return v;
 }
 
-// Exclusive scan over the 256 threads of a block; `sums` has 8 entries.
-__device__ __forceinline__ uint32_t block256_excl_scan(uint32_t v, uint32_t* sums, uint32_t* total) {
+// Exclusive scan over the NT threads of a block (NT a multiple of 32, at most 1024); `sums` has NT / 32 entries.
+template <int NT>
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* sums, uint32_t* total) {
     const int w = threadIdx.x >> 5;
     uint32_t incl = warp_incl_scan(v);
     if (sp_lane() == 31) sums[w] = incl;
     __syncthreads();
     uint32_t pre = 0, tot = 0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < NT / 32; ++i) {
         uint32_t s = sums[i];
         if (i < w) pre += s;
         tot += s;
@@ -174,6 +184,9 @@ __device__ __forceinline__ uint32_t block256_excl_scan(uint32_t v, uint32_t* sum
     __syncthreads();
     *total = tot;
     return incl - v + pre;
+}
+__device__ __forceinline__ uint32_t block256_excl_scan(uint32_t v, uint32_t* sums, uint32_t* total) {
+    return block_excl_scan<256>(v, sums, total);
 }
 
 // Tile histograms of one digit (passes after the first; the first pass's come from k_build_keys).
@@ -296,7 +309,7 @@ __device__ __forceinline__ void rank_rounds(const uint64_t (&key)[kSortIpt], int
 // the key's low bits; the last pass (split_bits >= 0) then separates the two again on the way out:
 // keys_out gets key >> split_bits, idx_out the low split_bits bits.
 template <bool PAY, int BITS>
-__global__ void __launch_bounds__(kSortThreads, 3)   // three tiles per SM hide the ranking chain's latency
+__global__ void __launch_bounds__(kSortThreads, SP_SORT_MIN_BLOCKS)   // several tiles per SM hide the ranking chain's latency
 k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict__ idx_in,
                  uint64_t* __restrict__ keys_out, uint32_t* __restrict__ idx_out, int64_t n, int shift,
                  const uint32_t* __restrict__ tilehist, int64_t ntiles,
@@ -309,7 +322,7 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
     uint32_t* wcnt = PAY ? sidx + kSortTile : sidx;           // [warps][RADIX + 1]
     uint32_t* dstart = wcnt + kSortWarps * (RADIX + 1);       // [RADIX + 1]
     uint32_t* goff = dstart + (RADIX + 1);                    // [RADIX]: global position of the digit's first key minus dstart (mod 2^32)
-    __shared__ uint32_t sums[8];
+    __shared__ uint32_t sums[kSortThreads / 32];
 
     const int t = threadIdx.x, w = t >> 5, lane = t & 31;
     const int64_t base = (int64_t)blockIdx.x * kSortTile;
@@ -364,8 +377,8 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
         }
     }
     uint32_t tot_all, gtot_all;
-    uint32_t ex = block256_excl_scan(mine, sums, &tot_all);
-    uint32_t gex = block256_excl_scan(gmine, sums, &gtot_all);
+    uint32_t ex = block_excl_scan<kSortThreads>(mine, sums, &tot_all);
+    uint32_t gex = block_excl_scan<kSortThreads>(gmine, sums, &gtot_all);
 #pragma unroll
     for (int q = 0; q < DPT; ++q) {
         const int d = t * DPT + q;
