@@ -227,27 +227,35 @@ def secondary_bounds(probes, torch, model):
     return out
 
 
-# Hit rates of the gather kernels' row loads, from single-launch ncu captures (profiles/): the share
-# of requested sectors served by L1, and of the L1 misses served by L2.  With them the gather bound is
-# max over levels of (bytes that must cross that level / the probed rate of that level): every
-# fetched row crosses the L1 data pipe, L1 misses cross L2 -> SM, L2 misses cross HBM -> L2.  None:
-# not captured for the current kernel; the bound then assumes no reuse at all (every row from the
-# level its table fits in).
-NCU_HIT = {
-    "spmm_dcsr": None, "spmm_csr": None, "sddmm_csr": None, "mttkrp_csf": None, "spmv_dcsr": None,
+# What each gather kernel moved at the three levels of the memory system in one launch at full size, from
+# single-launch ncu captures (profiles/; `bench.py --only-call NAME`): bytes through L2 (lts__t_bytes.sum)
+# and bytes from and to DRAM (dram__bytes_read.sum + dram__bytes_write.sum).  The bound of a launch is the
+# slowest of three transfers, each at the best rate measured for it in this same run:
+#   every gathered row crosses the L1 data pipe        gathered bytes / probe rate out of an L1-resident table
+#   what missed L1 crosses L2 -> SM                     L2 bytes       / probe rate out of an L2-resident table
+#   what missed L2 crosses HBM -> L2                    DRAM bytes     / measured copy bandwidth
+# A kernel cannot finish sooner than that with the locality it has.  None: the kernel has changed since
+# its capture; the bound then assumes no reuse (every row from the level its table fits in).
+NCU_LEVELS = {
+    "spmm_dcsr": None,
+    "spmv_dcsr": None,
+    "spmm_csr": {"lts_bytes": 0.656e9, "dram_bytes": 58.9e6, "source": "profiles/spmv_spmm_sddmm_full_configs.md"},
+    "sddmm_csr": {"lts_bytes": 3.147e9, "dram_bytes": 1.211e9, "source": "profiles/spmv_spmm_sddmm_full_configs.md"},
+    "mttkrp_csf": {"lts_bytes": 3.644e9, "dram_bytes": 0.2948e9, "source": "profiles/k_mttkrp_16384cube_20M.md"},
 }
 
 
-def gather_bound_ms(name, g, rates, table_bytes):
+def gather_bound_ms(name, g, rates, table_bytes, peak_gbs):
     nbytes = g["rows"] * g["row_elems"] * 8
-    hit = NCU_HIT.get(name)
-    if hit is None:
+    lv = NCU_LEVELS.get(name)
+    if lv is None:
         level = "l1" if table_bytes <= L1_TABLE_BYTES else ("l2" if table_bytes <= 64 << 20 else "hbm")
         return nbytes / (rates[level] * 1e9) * 1e3, f"no reuse, table in {level}"
-    l1_miss = 1.0 - hit["l1_hit"]
-    l2_miss = 1.0 - hit["l2_hit"]
-    t = max(nbytes / rates["l1"], nbytes * l1_miss / rates["l2"], nbytes * l1_miss * l2_miss / rates["hbm"])
-    return t / 1e9 * 1e3, f"L1 hit {hit['l1_hit']:.2f}, L2 hit {hit['l2_hit']:.2f} ({hit['source']})"
+    parts = {"l1": nbytes / (rates["l1"] * 1e9), "l2": lv["lts_bytes"] / (rates["l2"] * 1e9),
+             "hbm": lv["dram_bytes"] / (peak_gbs * 1e9)}
+    worst = max(parts, key=parts.get)
+    return parts[worst] * 1e3, (f"slowest level {worst}: L1 {parts['l1'] * 1e3:.3f} ms, L2 {parts['l2'] * 1e3:.3f} ms, "
+                                f"HBM {parts['hbm'] * 1e3:.3f} ms ({lv['source']})")
 
 
 # --------------------------------------------------------------------------- GPU arm
@@ -731,7 +739,7 @@ def main():
             # second bound: the rows the method fetches (one per stored entry) at the probed row-fetch rates
             g = m["gather"]
             rates = bounds["gather_gbs"][f"{g['row_elems'] * 8}B_rows"]
-            gms, how = gather_bound_ms(name, g, rates, g["table_rows"] * g["row_elems"] * 8)
+            gms, how = gather_bound_ms(name, g, rates, g["table_rows"] * g["row_elems"] * 8, peak)
             fms = m["flops"] / (bounds["dfma_tflops"] * 1e12) * 1e3
             kernels[name].update({"gather_bytes": g["rows"] * g["row_elems"] * 8, "gather_bound_ms": round(gms, 4),
                                   "gather_bound_model": how, "dfma_bound_ms": round(fms, 4),

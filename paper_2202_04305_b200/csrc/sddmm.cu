@@ -41,11 +41,8 @@ __device__ __forceinline__ void ld2(const double* p, double* a) {
 
 // NCH > 0: A[i,:] lives in NCH register chunks of 32*V columns (K <= NCH*32*V).
 // NCH == 0: any K, A is re-read (from L1) for every entry.
-#ifndef SP_LB_SDDMM
-#define SP_LB_SDDMM 1
-#endif
 template <typename P, typename I, int V, int NCH>
-__global__ void __launch_bounds__(kSThreads, SP_LB_SDDMM)
+__global__ void __launch_bounds__(kSThreads)
 k_sddmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ sval,
         const I* __restrict__ outer, const double* __restrict__ A, int64_t lda, const double* __restrict__ Bt,
         int64_t ldt, int64_t K, double* __restrict__ xv, const int64_t* __restrict__ prow,

@@ -22,11 +22,8 @@ constexpr int kVThreads = 256;
 constexpr int kVIpt = 8;
 constexpr int kVTile = kVThreads * kVIpt;   // merge items per CTA
 
-#ifndef SP_LB_SPMV
-#define SP_LB_SPMV 1
-#endif
 template <typename P, typename I, bool SCATTER>
-__global__ void __launch_bounds__(kVThreads, SP_LB_SPMV)
+__global__ void __launch_bounds__(kVThreads)
 k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
        const I* __restrict__ outer, const double* __restrict__ x, double* __restrict__ y,
        const int64_t* __restrict__ prow, const int64_t* __restrict__ pnz, int64_t nseg,
