@@ -232,26 +232,29 @@ def secondary_bounds(probes, torch, model):
 # and bytes from and to DRAM (dram__bytes_read.sum + dram__bytes_write.sum).  The bound of a launch is the
 # slowest of three transfers, each at the best rate measured for it in this same run:
 #   every gathered row crosses the L1 data pipe        gathered bytes / probe rate out of an L1-resident table
-#   what missed L1 crosses L2 -> SM                     L2 bytes       / probe rate out of an L2-resident table
+#   what missed L1 crosses L2 -> SM                     L2 bytes       / best probe rate out of an L2-resident table
 #   what missed L2 crosses HBM -> L2                    DRAM bytes     / measured copy bandwidth
 # A kernel cannot finish sooner than that with the locality it has.  None: the kernel has changed since
 # its capture; the bound then assumes no reuse (every row from the level its table fits in).
 NCU_LEVELS = {
-    "spmm_dcsr": None,
-    "spmv_dcsr": None,
+    "spmm_dcsr": {"lts_bytes": 2.394e9, "dram_bytes": 1.2056e9, "source": "profiles/spmv_spmm_sddmm_full_configs.md"},
+    "spmv_dcsr": {"lts_bytes": 331.7e6, "dram_bytes": 71.7e6, "source": "profiles/spmv_spmm_sddmm_full_configs.md"},
     "spmm_csr": {"lts_bytes": 0.656e9, "dram_bytes": 58.9e6, "source": "profiles/spmv_spmm_sddmm_full_configs.md"},
     "sddmm_csr": {"lts_bytes": 3.147e9, "dram_bytes": 1.211e9, "source": "profiles/spmv_spmm_sddmm_full_configs.md"},
     "mttkrp_csf": {"lts_bytes": 3.644e9, "dram_bytes": 0.2948e9, "source": "profiles/k_mttkrp_16384cube_20M.md"},
 }
 
 
-def gather_bound_ms(name, g, rates, table_bytes, peak_gbs):
+def gather_bound_ms(name, g, all_rates, table_bytes, peak_gbs):
     nbytes = g["rows"] * g["row_elems"] * 8
+    rates = dict(all_rates[f"{g['row_elems'] * 8}B_rows"])
     lv = NCU_LEVELS.get(name)
     if lv is None:
         level = "l1" if table_bytes <= L1_TABLE_BYTES else ("l2" if table_bytes <= 64 << 20 else "hbm")
         return nbytes / (rates[level] * 1e9) * 1e3, f"no reuse, table in {level}"
-    parts = {"l1": nbytes / (rates["l1"] * 1e9), "l2": lv["lts_bytes"] / (rates["l2"] * 1e9),
+    # L2 moves whole 32-byte sectors: the byte rate of the L2 level is the best one any row size reached
+    l2_rate = max(v["l2"] for v in all_rates.values())
+    parts = {"l1": nbytes / (rates["l1"] * 1e9), "l2": lv["lts_bytes"] / (l2_rate * 1e9),
              "hbm": lv["dram_bytes"] / (peak_gbs * 1e9)}
     worst = max(parts, key=parts.get)
     return parts[worst] * 1e3, (f"slowest level {worst}: L1 {parts['l1'] * 1e3:.3f} ms, L2 {parts['l2'] * 1e3:.3f} ms, "
@@ -738,8 +741,7 @@ def main():
         if "gather" in m:
             # second bound: the rows the method fetches (one per stored entry) at the probed row-fetch rates
             g = m["gather"]
-            rates = bounds["gather_gbs"][f"{g['row_elems'] * 8}B_rows"]
-            gms, how = gather_bound_ms(name, g, rates, g["table_rows"] * g["row_elems"] * 8, peak)
+            gms, how = gather_bound_ms(name, g, bounds["gather_gbs"], g["table_rows"] * g["row_elems"] * 8, peak)
             fms = m["flops"] / (bounds["dfma_tflops"] * 1e12) * 1e3
             kernels[name].update({"gather_bytes": g["rows"] * g["row_elems"] * 8, "gather_bound_ms": round(gms, 4),
                                   "gather_bound_model": how, "dfma_bound_ms": round(fms, 4),
@@ -816,8 +818,8 @@ def main():
 
 
 # DRAM bytes (read + write) per launch from ncu captures of the current kernels (profiles/): the sort's
-# scatter pass on 20,000,000 entries read 245.2 MB and wrote 220.0 MB (algorithmic: 480 MB; L2 absorbs the rest).
-NCU_TRAFFIC = {"k_sort_downsweep": 465.2e6}
+# scatter pass on 20,000,000 entries read 245.2 MB and wrote 221.7 MB (algorithmic: 480 MB; L2 absorbs the rest).
+NCU_TRAFFIC = {"k_sort_downsweep": 466.9e6}
 # one radix pass reads and writes a key (8 B) and an entry index (4 B) per entry
 SORT_PASS_BYTES_PER_ENTRY = 24
 

@@ -345,3 +345,32 @@ def test_mttkrp_any_output_mode(oracle, mode, R):
     with pytest.raises(b.SpError) as e:
         b.sp_mttkrp_mode(Tbad, mode, [dev(f) for f in F])
     assert e.value.code == 2
+
+
+def test_one_handle_on_two_streams(oracle):
+    """Calls on different streams share a handle: its cached tables are read-only once built and every
+    call's scratch (row carries) is its own.  Two streams run SpMM and SpMV over the same handle, merge
+    path and lane-group routes, with different operands, interleaved; both results must be right."""
+    import torch
+    for coo in (I.config2(seed=31, n=4000), I.config3(seed=32, n=1 << 12, nnz=40000)):
+        coords, vals = to_dev(coo)
+        A = sp().sp_pack(coo.dims, coords, vals, (0, 1))
+        m, n = coo.dims
+        Bs = [I.dense_operand(31, 10 + k, n, 32) for k in range(2)]
+        xs = [I.uniform_pm1(31, 20 + k, n) for k in range(2)]
+        refs = [oracle.spmm(m, coo.coords[0], coo.coords[1], coo.vals, B) for B in Bs]
+        yrefs = [oracle.spmv(m, coo.coords[0], coo.coords[1], coo.vals, x) for x in xs]
+        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        dB, dx = [dev(B) for B in Bs], [dev(x) for x in xs]
+        outs = [torch.empty(m, 32, dtype=torch.float64, device="cuda") for _ in range(2)]
+        ys = [torch.empty(m, dtype=torch.float64, device="cuda") for _ in range(2)]
+        torch.cuda.synchronize()
+        for rep in range(5):
+            for k, st in enumerate(streams):
+                with torch.cuda.stream(st):
+                    sp().sp_spmm(A, dB[k], outs[k])
+                    sp().sp_spmv(A, dx[k], ys[k])
+        torch.cuda.synchronize()
+        for k in range(2):
+            assert_close(outs[k].cpu().numpy(), refs[k][0], refs[k][1], f"stream {k} spmm")
+            assert_close(ys[k].cpu().numpy(), yrefs[k][0], yrefs[k][1], f"stream {k} spmv")
