@@ -818,8 +818,8 @@ def main():
 
 
 # DRAM bytes (read + write) per launch from ncu captures of the current kernels (profiles/): the sort's
-# scatter pass on 20,000,000 entries read 245.2 MB and wrote 221.7 MB (algorithmic: 480 MB; L2 absorbs the rest).
-NCU_TRAFFIC = {"k_sort_downsweep": 466.9e6}
+# scatter pass on 20,000,000 entries read 245.2 MB and wrote 191.5 MB (algorithmic: 480 MB; L2 absorbs the rest).
+NCU_TRAFFIC = {"k_sort_downsweep": 436.7e6}
 # one radix pass reads and writes a key (8 B) and an entry index (4 B) per entry
 SORT_PASS_BYTES_PER_ENTRY = 24
 

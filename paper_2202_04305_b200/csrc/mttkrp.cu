@@ -182,8 +182,16 @@ constexpr int kFastPer = 1024;   // entries per warp
 
 // A lane's S columns are S/2 pairs; pair n sits at column offset coff[n] of the 32-column tile,
 // laid out so that the lanes of a group read one contiguous run per 16-byte load.
-template <int S>
+// W256 (S = 4, all 32 columns in use, 32-byte aligned rows): the lane's four columns are adjacent and
+// come with one 32-byte load, which halves the load instructions and their address arithmetic.
+template <int S, bool W256>
 __device__ __forceinline__ void ld_cols(const double* p, const int* coff, double* a) {
+    if (W256) {
+        asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];"
+                     : "=d"(a[0]), "=d"(a[1]), "=d"(a[S > 2 ? 2 : 0]), "=d"(a[S > 3 ? 3 : 0])
+                     : "l"(p + coff[0]));
+        return;
+    }
 #pragma unroll
     for (int q = 0; q < S; q += 2) {
         const double2 t = *reinterpret_cast<const double2*>(p + coff[q / 2]);
@@ -195,7 +203,7 @@ __device__ __forceinline__ void ld_cols(const double* p, const int* coff, double
 #ifndef SP_LB_MTTKRP
 #define SP_LB_MTTKRP 2
 #endif
-template <typename P, typename I, int S>
+template <typename P, typename I, int S, bool W256>
 __global__ void __launch_bounds__(kTThreads, SP_LB_MTTKRP)
 k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* __restrict__ pos2,
               const I* __restrict__ crd1, const I* __restrict__ crd2, const double* __restrict__ val,
@@ -222,7 +230,7 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
         bool on[S / 2];
 #pragma unroll
         for (int n = 0; n < S / 2; ++n) {
-            const int c0 = n * 2 * GL + 2 * hl;
+            const int c0 = W256 ? 4 * hl + 2 * n : n * 2 * GL + 2 * hl;
             on[n] = rb + c0 < R;
             coff[n] = on[n] ? c0 : 0;          // idle lanes read column rb and never write
         }
@@ -298,8 +306,8 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
 #pragma unroll
                 for (int u = 0; u < kStepGroup; ++u) {
                     e[u] = mine[t0 + u];
-                    ld_cols<S>(F2g + e[u].koff, coff, c[u]);
-                    if (e[u].bw & 1u) ld_cols<S>(F1g + (e[u].bw >> 1), coff, b[u]);
+                    ld_cols<S, W256>(F2g + e[u].koff, coff, c[u]);
+                    if (e[u].bw & 1u) ld_cols<S, W256>(F1g + (e[u].bw >> 1), coff, b[u]);
                 }
 #pragma unroll
                 for (int u = 0; u < kStepGroup; ++u) {
@@ -361,7 +369,7 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
         if (g == 0) {
 #pragma unroll
             for (int q = 0; q < S; ++q) {
-                const int cc = (q / 2) * 2 * GL + 2 * hl + (q & 1);
+                const int cc = (W256 ? 4 * hl + 2 * (q / 2) : (q / 2) * 2 * GL + 2 * hl) + (q & 1);
                 s_car[2 * wi][cc] = head_v[q];
                 s_car[2 * wi + 1][cc] = tail_v[q];
             }
@@ -437,13 +445,17 @@ static sp_status mttkrp_levels(sp_tensor* T, const double* F1, const double* F2,
     if (st != SP_OK) return st;
     const unsigned blocks = (unsigned)sp_ceil_div(part.nchunks * 32, kTThreads);
     if (fast) {
-#define SP_MTTKRP_FAST(S)                                                                                              \
-    k_mttkrp_fast<P, I, S><<<blocks, kTThreads, 0, stream>>>(                                                          \
+#define SP_MTTKRP_FAST(S, W)                                                                                           \
+    k_mttkrp_fast<P, I, S, W><<<blocks, kTThreads, 0, stream>>>(                                                       \
         static_cast<const P*>(T->pos[1]), T->lt[0] == SP_COMPRESSED ? static_cast<const I*>(T->crd[0]) : nullptr,      \
         static_cast<const P*>(T->pos[2]), static_cast<const I*>(T->crd[1]), static_cast<const I*>(T->crd[2]), T->val,  \
         F1, F2, R, M, part.row, part.nz, part.aux, part.nchunks, T->npos[1] - 1, T->ncrd[1], T->dims[T->ord[0]], d1, d2)
+        // one 32-byte load per lane and factor row when every lane has its four columns and rows are 32-byte aligned
+        const bool w256 = R % 32 == 0 && reinterpret_cast<uintptr_t>(F1) % 32 == 0 && reinterpret_cast<uintptr_t>(F2) % 32 == 0;
         SP_DISPATCH_WIDTHS(T, {
-            if (R % 4 == 0) SP_MTTKRP_FAST(4); else SP_MTTKRP_FAST(2);
+            if (w256) SP_MTTKRP_FAST(4, true);
+            else if (R % 4 == 0) SP_MTTKRP_FAST(4, false);
+            else SP_MTTKRP_FAST(2, false);
         });
 #undef SP_MTTKRP_FAST
         SP_LAUNCH_CHECK();

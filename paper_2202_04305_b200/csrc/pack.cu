@@ -75,18 +75,18 @@ struct LevelPlan {
 // ------------------------------------------------------------------ keys ---
 struct LevelCoords { const void* p[SP_MAX_RANK]; };   // coordinate array of the dimension stored at level l
 
-#ifndef SP_SORT_THREADS
-#define SP_SORT_THREADS 256
-#endif
-#ifndef SP_SORT_IPT
-#define SP_SORT_IPT 16
-#endif
-#ifndef SP_SORT_MIN_BLOCKS
-#define SP_SORT_MIN_BLOCKS 3
-#endif
-constexpr int kSortThreads = SP_SORT_THREADS;
-constexpr int kSortIpt = SP_SORT_IPT;
-constexpr int kSortTile = kSortThreads * kSortIpt;   // 4096
+constexpr int kSortThreads = 256;
+// Sort tile: 256 threads x kIpt keys.  With a separate 32-bit payload (PAY: key and entry index as a
+// pair, 24 bytes moved per entry and pass) 8 keys per thread and four tiles per SM are the faster shape
+// (six scatter passes over 20,000,000 entries: 0.78 ms against 0.87 ms with 16 keys and three tiles);
+// with the index inside the key (8-byte words) 16 keys per thread and three tiles per SM are
+// (5,000,000 entries: pack 0.48 ms against 0.50 ms).  Every kernel of one sort uses the same shape.
+template <bool PAY>
+struct SortShape {
+    static constexpr int kIpt = PAY ? 8 : 16;
+    static constexpr int kTile = kSortThreads * kIpt;
+    static constexpr int kMinBlocks = PAY ? 4 : 3;
+};
 constexpr int kSortWarps = kSortThreads / 32;
 constexpr int kMaxRadix = 256;
 
@@ -95,10 +95,11 @@ constexpr int kMaxRadix = 256;
 // counting sweep of its own.
 // idx_bits > 0: the entry index rides in the low idx_bits bits of the key itself (the sort then
 // moves 8 bytes per entry instead of 12) and no index array is written.
-template <typename CT>
+template <typename CT, bool PAY>
 __global__ void __launch_bounds__(kSortThreads)
 k_build_keys(LevelCoords lc, int64_t n, LevelPlan p, uint64_t* keys, uint32_t* idx, int idx_bits, int* err,
              int shift0, uint32_t mask0, uint32_t* __restrict__ tilehist, int64_t ntiles) {
+    constexpr int kSortIpt = SortShape<PAY>::kIpt, kSortTile = SortShape<PAY>::kTile;
     __shared__ uint32_t hist[kSortWarps][kMaxRadix];
     const int t = threadIdx.x, w = t >> 5;
     for (int i = t; i < kSortWarps * kMaxRadix; i += kSortThreads) (&hist[0][0])[i] = 0;
@@ -109,7 +110,7 @@ k_build_keys(LevelCoords lc, int64_t n, LevelPlan p, uint64_t* keys, uint32_t* i
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
 #pragma unroll
-        for (int i = 0; i < kSortIpt / 2; ++i) {       // the loads of eight entries first
+        for (int i = 0; i < kSortIpt / 2; ++i) {       // the loads of half a thread's entries first
             const int64_t e = base + (int64_t)(half * (kSortIpt / 2) + i) * kSortThreads + t;
 #pragma unroll
             for (int l = 0; l < SP_MAX_RANK; ++l)
@@ -193,9 +194,10 @@ __device__ __forceinline__ uint32_t block256_excl_scan(uint32_t v, uint32_t* sum
 // Counting them inside the previous pass's scatter, with global atomics where the keys land, was
 // measured: skewed digits pile onto few counters and the 20,000,000-entry scatter went from 0.145 ms
 // to 0.59 ms per pass.
-template <int BITS>
+template <int BITS, bool PAY>
 __global__ void __launch_bounds__(kSortThreads)
 k_sort_upsweep(const uint64_t* __restrict__ keys, int64_t n, int shift, uint32_t* __restrict__ tilehist, int64_t ntiles) {
+    constexpr int kSortIpt = SortShape<PAY>::kIpt, kSortTile = SortShape<PAY>::kTile;
     constexpr int RADIX = 1 << BITS;
     constexpr uint32_t mask = RADIX - 1;
     __shared__ uint32_t hist[kSortWarps][RADIX];     // one histogram per warp: conflicts only inside a warp
@@ -239,53 +241,69 @@ __device__ __forceinline__ uint32_t same_value_lanes(uint32_t d) {
     return peers;
 }
 
-// One block per digit: exclusive scan of that digit's tile counts, in place.  The counts are staged
-// in shared memory with coalesced loads; a thread then scans a contiguous run of them, and one block
-// scan joins the runs.
-constexpr int kScanChunk = 8192;
+// Exclusive scan of every digit's tile counts, in place, in two small launches: the counts of a digit
+// are cut into chunks of kScanChunk tiles; k_sort_chunk_totals adds up each chunk, k_sort_scan scans a
+// chunk starting from the sum of the chunks before it (a handful of values, added up by every block
+// for itself).  Grid (digits, chunks): all SMs take part however many tiles there are.
+constexpr int kScanChunk = 2048;
 
 __global__ void __launch_bounds__(256)
-k_sort_scan(uint32_t* tilehist, int64_t ntiles, uint32_t* digit_total) {
+k_sort_chunk_totals(const uint32_t* __restrict__ tilehist, int64_t ntiles, int64_t nchunks, uint32_t* __restrict__ chunk_tot) {
+    __shared__ uint32_t sums[8];
+    const uint32_t* row = tilehist + (int64_t)blockIdx.x * ntiles;
+    const int64_t base = (int64_t)blockIdx.y * kScanChunk;
+    uint32_t local = 0;
+#pragma unroll
+    for (int i = 0; i < kScanChunk / 256; ++i) {
+        const int64_t q = base + i * 256 + threadIdx.x;
+        if (q < ntiles) local += row[q];
+    }
+    uint32_t tot;
+    block256_excl_scan(local, sums, &tot);
+    if (threadIdx.x == 0) chunk_tot[(int64_t)blockIdx.x * nchunks + blockIdx.y] = tot;
+}
+
+__global__ void __launch_bounds__(256)
+k_sort_scan(uint32_t* tilehist, int64_t ntiles, int64_t nchunks, const uint32_t* __restrict__ chunk_tot,
+            uint32_t* __restrict__ digit_total) {
     __shared__ uint32_t stage[kScanChunk];
     __shared__ uint32_t sums[8];
     uint32_t* row = tilehist + (int64_t)blockIdx.x * ntiles;
+    const int64_t base = (int64_t)blockIdx.y * kScanChunk;
+    const int cnt = (int)min((int64_t)kScanChunk, ntiles - base);
     constexpr int kPer = kScanChunk / 256;
-    uint32_t carry = 0;
-    for (int64_t base = 0; base < ntiles; base += kScanChunk) {
-        const int cnt = (int)min((int64_t)kScanChunk, ntiles - base);
-        for (int i = threadIdx.x; i < cnt; i += 256) stage[i] = row[base + i];
-        __syncthreads();
-        uint32_t local = 0;
+    uint32_t before = 0;                               // sum of the chunks before this one
+    for (int64_t c = 0; c < (int64_t)blockIdx.y; ++c) before += chunk_tot[(int64_t)blockIdx.x * nchunks + c];
+    for (int i = threadIdx.x; i < cnt; i += 256) stage[i] = row[base + i];
+    __syncthreads();
+    uint32_t local = 0;
 #pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            const int q = threadIdx.x * kPer + i;
-            if (q < cnt) local += stage[q];
-        }
-        uint32_t tot;
-        uint32_t run = block256_excl_scan(local, sums, &tot) + carry;
-#pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            const int q = threadIdx.x * kPer + i;
-            if (q < cnt) { const uint32_t v = stage[q]; stage[q] = run; run += v; }
-        }
-        __syncthreads();
-        for (int i = threadIdx.x; i < cnt; i += 256) row[base + i] = stage[i];
-        __syncthreads();
-        carry += tot;
+    for (int i = 0; i < kPer; ++i) {
+        const int q = threadIdx.x * kPer + i;
+        if (q < cnt) local += stage[q];
     }
-    if (threadIdx.x == 0) digit_total[blockIdx.x] = carry;
+    uint32_t tot;
+    uint32_t run = block256_excl_scan(local, sums, &tot) + before;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+        const int q = threadIdx.x * kPer + i;
+        if (q < cnt) { const uint32_t v = stage[q]; stage[q] = run; run += v; }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < cnt; i += 256) row[base + i] = stage[i];
+    if (threadIdx.x == 0 && blockIdx.y == nchunks - 1) digit_total[blockIdx.x] = before + tot;
 }
 
 constexpr size_t down_smem(bool pay, int bits) {
-    return (size_t)kSortTile * 8 + (pay ? (size_t)kSortTile * 4 : 0) + (size_t)kSortWarps * ((1 << bits) + 1) * 4 +
+    return (size_t)(pay ? SortShape<true>::kTile : SortShape<false>::kTile) * (pay ? 12 : 8) + (size_t)kSortWarps * ((1 << bits) + 1) * 4 +
            (size_t)((1 << bits) + 1) * 4 + (size_t)(1 << bits) * 4 + 64;
 }
 
-// Ranks the warp's 16 rounds of 32 keys: rank i = number of earlier keys of this warp with the same
+// Ranks the warp's rounds of 32 keys: rank i = number of earlier keys of this warp with the same
 // digit (below 512, so two ranks share a register: round i sits in half i & 1 of rank[i / 2]); the
 // per-warp digit counts end up in mycnt[].  NB = BITS, or BITS + 1 when the tile has padding slots
 // (their digit is RADIX, which sorts after every real digit).
-template <int BITS, int NB>
+template <int BITS, int NB, int kSortIpt>
 __device__ __forceinline__ void rank_rounds(const uint64_t (&key)[kSortIpt], int shift, int w, int lane, int tile_n,
                                             uint32_t* mycnt, uint32_t (&rank)[kSortIpt / 2]) {
     constexpr uint32_t RADIX = 1u << BITS;
@@ -309,11 +327,12 @@ __device__ __forceinline__ void rank_rounds(const uint64_t (&key)[kSortIpt], int
 // the key's low bits; the last pass (split_bits >= 0) then separates the two again on the way out:
 // keys_out gets key >> split_bits, idx_out the low split_bits bits.
 template <bool PAY, int BITS>
-__global__ void __launch_bounds__(kSortThreads, SP_SORT_MIN_BLOCKS)   // several tiles per SM hide the ranking chain's latency
+__global__ void __launch_bounds__(kSortThreads, SortShape<PAY>::kMinBlocks)   // several tiles per SM hide the ranking chain's latency
 k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict__ idx_in,
                  uint64_t* __restrict__ keys_out, uint32_t* __restrict__ idx_out, int64_t n, int shift,
                  const uint32_t* __restrict__ tilehist, int64_t ntiles,
                  const uint32_t* __restrict__ digit_total, int split_bits) {
+    constexpr int kSortIpt = SortShape<PAY>::kIpt, kSortTile = SortShape<PAY>::kTile;
     constexpr int RADIX = 1 << BITS;
     constexpr uint32_t mask = RADIX - 1;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -342,8 +361,8 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
         key[i] = valid ? keys_in[base + li] : 0;
         pay[i] = (PAY && valid) ? idx_in[base + li] : 0;
     }
-    if (tile_n == kSortTile) rank_rounds<BITS, BITS>(key, shift, w, lane, tile_n, mycnt, rank);
-    else rank_rounds<BITS, BITS + 1>(key, shift, w, lane, tile_n, mycnt, rank);
+    if (tile_n == kSortTile) rank_rounds<BITS, BITS, kSortIpt>(key, shift, w, lane, tile_n, mycnt, rank);
+    else rank_rounds<BITS, BITS + 1, kSortIpt>(key, shift, w, lane, tile_n, mycnt, rank);
     __syncthreads();
 
     // per digit: exclusive scan over warps; then exclusive scan over digits (each thread owns
@@ -425,14 +444,23 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
 // digit of BITS bits at `shift`.
 template <int BITS>
 sp_status sort_pass(const uint64_t* kin, const uint32_t* iin, uint64_t* kout, uint32_t* iout, int64_t n, int shift,
-                    uint32_t* tilehist, int64_t stiles, uint32_t* digit_total, bool fused, int split_bits,
+                    uint32_t* tilehist, int64_t stiles, uint32_t* digit_total, uint32_t* chunk_tot, bool fused, int split_bits,
                     bool have_hist, cudaStream_t stream, PhaseTimer& timer) {
     if (!have_hist) {
-        k_sort_upsweep<BITS><<<(unsigned)stiles, kSortThreads, 0, stream>>>(kin, n, shift, tilehist, stiles);
+        if (fused) k_sort_upsweep<BITS, false><<<(unsigned)stiles, kSortThreads, 0, stream>>>(kin, n, shift, tilehist, stiles);
+        else k_sort_upsweep<BITS, true><<<(unsigned)stiles, kSortThreads, 0, stream>>>(kin, n, shift, tilehist, stiles);
         sp_count_launches(1);
     }
     timer.mark(kPhUpsweep);
-    k_sort_scan<<<1 << BITS, 256, 0, stream>>>(tilehist, stiles, digit_total);
+    {
+        const int64_t nchunks = sp_ceil_div(stiles, kScanChunk);
+        dim3 grid(1u << BITS, (unsigned)nchunks);
+        if (nchunks > 1) {
+            k_sort_chunk_totals<<<grid, 256, 0, stream>>>(tilehist, stiles, nchunks, chunk_tot);
+            sp_count_launches(1);
+        }
+        k_sort_scan<<<grid, 256, 0, stream>>>(tilehist, stiles, nchunks, chunk_tot, digit_total);
+    }
     timer.mark(kPhScan);
     if (fused) {
         SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep<false, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -836,9 +864,15 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         uint64_t* kbuf[2] = {ws.get<uint64_t>((size_t)n), ws.get<uint64_t>((size_t)n)};
         uint32_t* ibuf[2] = {ws.get<uint32_t>((size_t)n), ws.get<uint32_t>((size_t)n)};
         d_err = ws.get<int>(1);
-        const int64_t stiles = sp_ceil_div(n, kSortTile);
+        const int npasses = (total_bits + kMaxDigitBits - 1) / kMaxDigitBits;
+        // the entry index rides inside the key when both fit in 64 bits
+        int idx_bits = 0;
+        while (((int64_t)1 << idx_bits) < n) ++idx_bits;
+        const bool fused = npasses > 0 && idx_bits > 0 && total_bits + idx_bits <= 64;
+        const int64_t stiles = sp_ceil_div(n, fused ? SortShape<false>::kTile : SortShape<true>::kTile);
         uint32_t* tilehist = ws.get<uint32_t>((size_t)stiles << kMaxDigitBits);
         uint32_t* digit_total = ws.get<uint32_t>((size_t)1 << kMaxDigitBits);
+        uint32_t* chunk_tot = ws.get<uint32_t>((size_t)sp_ceil_div(stiles, kScanChunk) << kMaxDigitBits);
         ct_tiles = sp_ceil_div(n, kCtTile);
         uint64_t* tilesum = ws.get<uint64_t>((size_t)ct_tiles);
         tileprefix = ws.get<int64_t>((size_t)ct_tiles * SP_MAX_RANK);
@@ -848,11 +882,6 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
 
         LevelCoords lc;
         for (int l = 0; l < SP_MAX_RANK; ++l) lc.p[l] = coo_coords[l < rank ? plan.src[l] : 0];
-        const int npasses = (total_bits + kMaxDigitBits - 1) / kMaxDigitBits;
-        // the entry index rides inside the key when both fit in 64 bits
-        int idx_bits = 0;
-        while (((int64_t)1 << idx_bits) < n) ++idx_bits;
-        const bool fused = npasses > 0 && idx_bits > 0 && total_bits + idx_bits <= 64;
         // digit widths as even as possible, the wider ones first
         int widths[16], shifts[16];
         for (int ps = 0, kshift = 0; ps < npasses; ++ps) {
@@ -863,12 +892,12 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         }
         const int shift0 = npasses ? shifts[0] : 0;
         const uint32_t mask0 = npasses ? (1u << widths[0]) - 1u : 0u;
-        if (coo_coord_bits == 32)
-            k_build_keys<int32_t><<<(unsigned)stiles, kSortThreads, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], fused ? idx_bits : 0,
-                                                                              d_err, shift0, mask0, tilehist, stiles);
-        else
-            k_build_keys<int64_t><<<(unsigned)stiles, kSortThreads, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], fused ? idx_bits : 0,
-                                                                              d_err, shift0, mask0, tilehist, stiles);
+#define SP_BUILD_KEYS(CT, PAY)                                                                                       \
+    k_build_keys<CT, PAY><<<(unsigned)stiles, kSortThreads, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], fused ? idx_bits : 0, \
+                                                                        d_err, shift0, mask0, tilehist, stiles)
+        if (coo_coord_bits == 32) { if (fused) SP_BUILD_KEYS(int32_t, false); else SP_BUILD_KEYS(int32_t, true); }
+        else { if (fused) SP_BUILD_KEYS(int64_t, false); else SP_BUILD_KEYS(int64_t, true); }
+#undef SP_BUILD_KEYS
         SP_LAUNCH_CHECK();
         sp_count_launches(1);
         timer.mark(kPhKeys);
@@ -880,7 +909,7 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
 #define SP_SORT_PASS(B)                                                                                             \
     case B:                                                                                                         \
         ps_st = sort_pass<B>(kbuf[cur], ibuf[cur], kbuf[cur ^ 1], ibuf[cur ^ 1], n, shifts[ps], tilehist, stiles,    \
-                             digit_total, fused, split, ps == 0, stream, timer);                                     \
+                             digit_total, chunk_tot, fused, split, ps == 0, stream, timer);                          \
         break;
             switch (widths[ps]) {
                 SP_SORT_PASS(1) SP_SORT_PASS(2) SP_SORT_PASS(3) SP_SORT_PASS(4) SP_SORT_PASS(5)
