@@ -68,8 +68,8 @@ typedef enum {
     SP_ERR_DUPLICATE = 5,       /* SP_DUP_ERROR was set and two entries share coordinates */
     SP_ERR_ALLOC = 6,           /* the allocator returned NULL */
     SP_ERR_CUDA = 7,            /* a CUDA runtime call failed */
-    SP_ERR_TIMEOUT = 8,         /* reserved (a bounded device-side wait ran out): no kernel here waits on
-                                   another, so no call returns it */
+    SP_ERR_TIMEOUT = 8,         /* a bounded device-side wait ran out: an earlier sp_spmm launch whose operand
+                                   tiles arrive by asynchronous copy gave up waiting for one; see sp_spmm */
     SP_ERR_TOO_LARGE = 9        /* the problem does not fit a fixed-capacity entry point (sp_spmv_static) */
 } sp_status;
 
@@ -182,8 +182,15 @@ sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* stream);
  * f64 matrix instruction (the one place in this library where tensor cores
  * apply; the sparse kernels are gathers and use none); when it has few output
  * rows its contraction index is split over thread blocks and the partial sums
- * meet in C through atomics too (row-major included).  A column-major matrix
- * with 2^32 or more columns is refused (SP_ERR_UNSUPPORTED).
+ * meet in C through atomics too (row-major included).  Row-major, with the
+ * stored slices and every row of B starting on 16-byte boundaries (even slice
+ * length, even ldb, aligned pointers), the operand tiles are brought in by the
+ * copy engine (tensor maps over this device's memory, built per call on the
+ * host); otherwise threads stage them.  The kernel's waits for those copies
+ * are bounded: if one runs out, the blocks concerned write nothing, a flag is
+ * raised, and this and every later such call returns SP_ERR_TIMEOUT instead of
+ * launching (the contents of that earlier C are then undefined).  A
+ * column-major matrix with 2^32 or more columns is refused (SP_ERR_UNSUPPORTED).
  */
 sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t ldb,
                   double* C, int64_t ldc, void* stream);

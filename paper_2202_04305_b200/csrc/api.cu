@@ -53,7 +53,7 @@ const char* sp_status_string(sp_status s) {
         case SP_ERR_DUPLICATE: return "duplicate coordinates";
         case SP_ERR_ALLOC: return "device allocation failed";
         case SP_ERR_CUDA: return "CUDA runtime error";
-        case SP_ERR_TIMEOUT: return "bounded device-side wait ran out (reserved: no call returns it)";
+        case SP_ERR_TIMEOUT: return "a bounded device-side wait for an asynchronous copy ran out in an earlier launch";
         case SP_ERR_TOO_LARGE: return "problem exceeds the fixed scratch capacity of this entry point";
     }
     return "unknown status";

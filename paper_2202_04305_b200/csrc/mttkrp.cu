@@ -288,13 +288,15 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
             st.koff = valid ? (uint32_t)SP_IDX(k_l, d2) * Ru : 0u;
             st.bw = valid ? (((j * Ru) << 1) | (close ? 1u : 0u)) : 0u;
             st.v = valid ? v_l : 0.0;
-            s_st[wi][lane] = st;
+            // entry e = g * GL + t is parked at slot t * S + g: the S groups read step t's entries from one
+            // 16 * S-byte run (one shared-memory wavefront, where slots g * GL + t cost S: same banks)
+            s_st[wi][(lane % GL) * S + lane / GL] = st;
             __syncwarp();
 
             double accf[S];
 #pragma unroll
             for (int q = 0; q < S; ++q) accf[q] = 0.0;
-            const Staged* mine = &s_st[wi][g * GL];
+            const Staged* mine = &s_st[wi][g];
 #pragma unroll
             for (int t0 = 0; t0 < GL; t0 += kStepGroup) {
                 // Note: no double is set to a constant zero in this loop.  Zeroing a 64-bit register
@@ -305,7 +307,7 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
                 double c[kStepGroup][S], b[kStepGroup][S];
 #pragma unroll
                 for (int u = 0; u < kStepGroup; ++u) {
-                    e[u] = mine[t0 + u];
+                    e[u] = mine[(t0 + u) * S];
                     ld_cols<S, W256>(F2g + e[u].koff, coff, c[u]);
                     if (e[u].bw & 1u) ld_cols<S, W256>(F1g + (e[u].bw >> 1), coff, b[u]);
                 }

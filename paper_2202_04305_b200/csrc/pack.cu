@@ -579,7 +579,12 @@ struct EmitArgs {
     int* err;
 };
 
-__global__ void __launch_bounds__(kCtThreads) k_emit(EmitArgs a) {
+#ifdef SP_LB_EMIT
+#define SP_EMIT_BOUNDS __launch_bounds__(kCtThreads, SP_LB_EMIT)
+#else
+#define SP_EMIT_BOUNDS __launch_bounds__(kCtThreads)
+#endif
+__global__ void SP_EMIT_BOUNDS k_emit(EmitArgs a) {
     __shared__ uint64_t sums[16];
     const LevelPlan& p = a.plan;
     const int64_t e0 = (int64_t)blockIdx.x * kCtTile + (int64_t)threadIdx.x * kCtIpt;

@@ -257,8 +257,13 @@ __device__ __forceinline__ void st_vec(double* p, const double* a) {
 // bit comes up (rows without entries that end at the same place are stored as zeros).
 constexpr int kGather = 8;
 
+#ifdef SP_LB_GATHER
+#define SP_GATHER_BOUNDS __launch_bounds__(kMThreads, SP_LB_GATHER)
+#else
+#define SP_GATHER_BOUNDS __launch_bounds__(kMThreads)
+#endif
 template <typename P, typename I, int V>
-__global__ void __launch_bounds__(kMThreads)
+__global__ void SP_GATHER_BOUNDS
 k_spmm_gather(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
               const I* __restrict__ outer, const double* __restrict__ B, int64_t N, int64_t ldb,
               double* __restrict__ C, int64_t ldc, const int64_t* __restrict__ prow,
@@ -362,8 +367,13 @@ k_spmm_gather(const P* __restrict__ pos, const I* __restrict__ crd, const double
 #ifndef SP_SPMM_ROWS_THREADS
 #define SP_SPMM_ROWS_THREADS 256
 #endif
+#ifdef SP_LB_ROWS
+#define SP_ROWS_BOUNDS __launch_bounds__(SP_SPMM_ROWS_THREADS, SP_LB_ROWS)
+#else
+#define SP_ROWS_BOUNDS __launch_bounds__(SP_SPMM_ROWS_THREADS)
+#endif
 template <typename P, typename I, int L, int V>
-__global__ void __launch_bounds__(SP_SPMM_ROWS_THREADS)
+__global__ void SP_ROWS_BOUNDS
 k_spmm_rows(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
             const I* __restrict__ outer, const double* __restrict__ B, int64_t ldb, double* __restrict__ C,
             int64_t ldc, int64_t nseg, int64_t m, int64_t n) {

@@ -75,6 +75,34 @@ def test_spmm_dense_inner_level(oracle, enc, N, name, coo):
     assert_close(Cg, ref, bd, f"spmm {enc} {name} N={N}")
 
 
+@pytest.mark.parametrize("m,n,nnz,N,ldb,shift,cbits", [
+    (700, 518, 60000, 50, 52, 0, 32),      # ragged rows, k and columns; padded B: copy-engine feed
+    (700, 518, 60000, 50, 52, 1, 32),      # B starts 8 bytes off a 16-byte boundary: register-staged feed
+    (700, 517, 60000, 32, 32, 0, 32),      # odd slice length: register-staged feed
+    (300, 20000, 90000, 32, 32, 0, 64),    # few rows, long contraction: split over k, 64-bit coordinates
+    (40, 30, 500, 8, 8, 0, 32),            # smaller than one tile in every direction
+])
+@pytest.mark.parametrize("lt", [(1, 0), (0, 0)])
+def test_spmm_dense_inner_both_feeds(oracle, m, n, nnz, N, ldb, shift, cbits, lt):
+    """Row-major products over a dense inner level run on the tensor-memory-accelerator feed when
+    every row of the stored slices and of B starts on a 16-byte boundary, and on the register-staged
+    kernel otherwise; both must agree with the oracle, ignore what lies beyond B's N columns and leave
+    the other columns of a strided C alone."""
+    import torch
+    coo = I.uniform_matrix(m, n, nnz, seed=31)
+    B = I.dense_operand(31, 3, n, N)
+    ref, bd = oracle.spmm(m, coo.coords[0], coo.coords[1], coo.vals, B)
+    coords, vals = to_dev(coo, cbits)
+    A = sp().sp_pack(coo.dims, coords, vals, lt, (0, 1), 32, cbits)
+    flat = torch.full((n * ldb + 2,), 1e300, dtype=torch.float64, device="cuda")
+    Bdev = flat[shift:shift + n * ldb].view(n, ldb)[:, :N]
+    Bdev.copy_(dev(B))
+    Cbig = torch.full((m, N + 3), 7.0, dtype=torch.float64, device="cuda")
+    sp().sp_spmm(A, Bdev, Cbig[:, :N])
+    assert_close(Cbig[:, :N].cpu().numpy(), ref, bd, "dense inner")
+    assert torch.all(Cbig[:, N:] == 7.0)
+
+
 @pytest.mark.parametrize("enc", list(MATRIX_ENCODINGS))
 @pytest.mark.parametrize("N", [1, 5, 32, 64, 70])
 @pytest.mark.parametrize("name,coo", MATS, ids=[m[0] for m in MATS])
