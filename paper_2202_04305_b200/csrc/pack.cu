@@ -94,10 +94,11 @@ constexpr int kMaxRadix = 256;
 // histogram for the first radix pass (digit = (key >> shift0) & mask0), so that pass needs no
 // counting sweep of its own.
 // idx_bits > 0: the entry index rides in the low idx_bits bits of the key itself (the sort then
-// moves 8 bytes per entry instead of 12) and no index array is written.
+// moves 8 bytes per entry).  Otherwise the entry's value travels beside its key from the first
+// pass on (which reads it from the input, where value e belongs to key e), so no index exists.
 template <typename CT, bool PAY>
 __global__ void __launch_bounds__(kSortThreads)
-k_build_keys(LevelCoords lc, int64_t n, LevelPlan p, uint64_t* keys, uint32_t* idx, int idx_bits, int* err,
+k_build_keys(LevelCoords lc, int64_t n, LevelPlan p, uint64_t* keys, int idx_bits, int* err,
              int shift0, uint32_t mask0, uint32_t* __restrict__ tilehist, int64_t ntiles) {
     constexpr int kSortIpt = SortShape<PAY>::kIpt, kSortTile = SortShape<PAY>::kTile;
     __shared__ uint32_t hist[kSortWarps][kMaxRadix];
@@ -129,11 +130,7 @@ k_build_keys(LevelCoords lc, int64_t n, LevelPlan p, uint64_t* keys, uint32_t* i
                     key |= (uint64_t)v << p.shift[l];
                 }
             }
-            if (idx_bits > 0) {
-                key = (key << idx_bits) | (uint64_t)e;
-            } else {
-                idx[e] = (uint32_t)e;
-            }
+            if (idx_bits > 0) key = (key << idx_bits) | (uint64_t)e;
             keys[e] = key;
             atomicAdd(&hist[w][(uint32_t)(key >> shift0) & mask0], 1u);
         }
@@ -295,7 +292,7 @@ k_sort_scan(uint32_t* tilehist, int64_t ntiles, int64_t nchunks, const uint32_t*
 }
 
 constexpr size_t down_smem(bool pay, int bits) {
-    return (size_t)(pay ? SortShape<true>::kTile : SortShape<false>::kTile) * (pay ? 12 : 8) + (size_t)kSortWarps * ((1 << bits) + 1) * 4 +
+    return (size_t)(pay ? SortShape<true>::kTile : SortShape<false>::kTile) * (pay ? 16 : 8) + (size_t)kSortWarps * ((1 << bits) + 1) * 4 +
            (size_t)((1 << bits) + 1) * 4 + (size_t)(1 << bits) * 4 + 64;
 }
 
@@ -323,13 +320,14 @@ __device__ __forceinline__ void rank_rounds(const uint64_t (&key)[kSortIpt], int
     }
 }
 
-// PAY: a 32-bit payload (the entry index) travels beside every key.  Without it the index sits in
-// the key's low bits; the last pass (split_bits >= 0) then separates the two again on the way out:
-// keys_out gets key >> split_bits, idx_out the low split_bits bits.
+// PAY: a 64-bit payload (the entry's value, moved as bits) travels beside every key.  Without it the
+// entry index sits in the key's low bits; the last pass (split_bits >= 0) then separates the two again
+// on the way out: keys_out gets key >> split_bits, idx_out the low split_bits bits.
 template <bool PAY, int BITS>
 __global__ void __launch_bounds__(kSortThreads, SortShape<PAY>::kMinBlocks)   // several tiles per SM hide the ranking chain's latency
-k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict__ idx_in,
-                 uint64_t* __restrict__ keys_out, uint32_t* __restrict__ idx_out, int64_t n, int shift,
+k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint64_t* __restrict__ pay_in,
+                 uint64_t* __restrict__ keys_out, uint64_t* __restrict__ pay_out, uint32_t* __restrict__ idx_out,
+                 int64_t n, int shift,
                  const uint32_t* __restrict__ tilehist, int64_t ntiles,
                  const uint32_t* __restrict__ digit_total, int split_bits) {
     constexpr int kSortIpt = SortShape<PAY>::kIpt, kSortTile = SortShape<PAY>::kTile;
@@ -337,8 +335,8 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
     constexpr uint32_t mask = RADIX - 1;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t* skeys = reinterpret_cast<uint64_t*>(smem_raw);
-    uint32_t* sidx = reinterpret_cast<uint32_t*>(skeys + kSortTile);
-    uint32_t* wcnt = PAY ? sidx + kSortTile : sidx;           // [warps][RADIX + 1]
+    uint64_t* spay = skeys + kSortTile;
+    uint32_t* wcnt = reinterpret_cast<uint32_t*>(PAY ? spay + kSortTile : spay);   // [warps][RADIX + 1]
     uint32_t* dstart = wcnt + kSortWarps * (RADIX + 1);       // [RADIX + 1]
     uint32_t* goff = dstart + (RADIX + 1);                    // [RADIX]: global position of the digit's first key minus dstart (mod 2^32)
     __shared__ uint32_t sums[kSortThreads / 32];
@@ -351,18 +349,25 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
     __syncthreads();
 
     uint64_t key[kSortIpt];
-    uint32_t pay[kSortIpt];
+    uint64_t pay[PAY ? kSortIpt : 1];
     uint32_t rank[kSortIpt / 2];
     uint32_t* mycnt = wcnt + w * (RADIX + 1);
 #pragma unroll
-    for (int i = 0; i < kSortIpt; ++i) {             // all loads first
+    for (int i = 0; i < kSortIpt; ++i) {             // all key loads first
         const int li = w * (32 * kSortIpt) + i * 32 + lane;
-        const bool valid = li < tile_n;
-        key[i] = valid ? keys_in[base + li] : 0;
-        pay[i] = (PAY && valid) ? idx_in[base + li] : 0;
+        key[i] = li < tile_n ? keys_in[base + li] : 0;
     }
     if (tile_n == kSortTile) rank_rounds<BITS, BITS, kSortIpt>(key, shift, w, lane, tile_n, mycnt, rank);
     else rank_rounds<BITS, BITS + 1, kSortIpt>(key, shift, w, lane, tile_n, mycnt, rank);
+    if (PAY) {
+        // the payloads are not needed before the exchange: requested here, they arrive during the
+        // digit scans below without holding registers through the ranking
+#pragma unroll
+        for (int i = 0; i < kSortIpt; ++i) {
+            const int li = w * (32 * kSortIpt) + i * 32 + lane;
+            pay[i] = li < tile_n ? pay_in[base + li] : 0;
+        }
+    }
     __syncthreads();
 
     // per digit: exclusive scan over warps; then exclusive scan over digits (each thread owns
@@ -420,7 +425,7 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
         const uint32_t s = dstart[d] + mycnt[d] + ((i & 1) ? rank[i / 2] >> 16 : rank[i / 2] & 0xffffu);
         if (valid) {
             skeys[s] = key[i];
-            if (PAY) sidx[s] = pay[i];
+            if (PAY) spay[s] = pay[i];
         }
     }
     __syncthreads();
@@ -430,7 +435,7 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
         const uint32_t o = goff[d] + (uint32_t)s;
         if (PAY) {
             keys_out[o] = k;
-            idx_out[o] = sidx[s];
+            pay_out[o] = spay[s];
         } else if (split_bits >= 0) {
             keys_out[o] = split_bits < 64 ? k >> split_bits : 0;
             idx_out[o] = (uint32_t)(k & ((1ull << split_bits) - 1ull));
@@ -443,7 +448,7 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint32_t* __restric
 // One radix pass (tile histograms unless they exist already, per-digit scans, ranked scatter) for a
 // digit of BITS bits at `shift`.
 template <int BITS>
-sp_status sort_pass(const uint64_t* kin, const uint32_t* iin, uint64_t* kout, uint32_t* iout, int64_t n, int shift,
+sp_status sort_pass(const uint64_t* kin, const uint64_t* pin, uint64_t* kout, uint64_t* pout, uint32_t* iout, int64_t n, int shift,
                     uint32_t* tilehist, int64_t stiles, uint32_t* digit_total, uint32_t* chunk_tot, bool fused, int split_bits,
                     bool have_hist, cudaStream_t stream, PhaseTimer& timer) {
     if (!have_hist) {
@@ -466,12 +471,12 @@ sp_status sort_pass(const uint64_t* kin, const uint32_t* iin, uint64_t* kout, ui
         SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep<false, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)down_smem(false, BITS)));
         k_sort_downsweep<false, BITS><<<(unsigned)stiles, kSortThreads, down_smem(false, BITS), stream>>>(
-            kin, nullptr, kout, iout, n, shift, tilehist, stiles, digit_total, split_bits);
+            kin, nullptr, kout, nullptr, iout, n, shift, tilehist, stiles, digit_total, split_bits);
     } else {
         SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep<true, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)down_smem(true, BITS)));
         k_sort_downsweep<true, BITS><<<(unsigned)stiles, kSortThreads, down_smem(true, BITS), stream>>>(
-            kin, iin, kout, iout, n, shift, tilehist, stiles, digit_total, -1);
+            kin, pin, kout, pout, nullptr, n, shift, tilehist, stiles, digit_total, -1);
     }
     SP_LAUNCH_CHECK();
     timer.mark(kPhDownsweep);
@@ -485,14 +490,6 @@ constexpr int kCtIpt = 8;
 constexpr int kCtTile = kCtThreads * kCtIpt;   // 2048
 constexpr int kField = 12;                     // SP_MAX_RANK 12-bit counters (a tile has 2048 entries) in 64 bits
 constexpr uint64_t kFieldMask = (1ull << kField) - 1;
-
-__device__ __forceinline__ uint64_t level_flags(uint64_t k, uint64_t kprev, bool first, const LevelPlan& p) {
-    uint64_t x = k ^ kprev, f = 0;
-#pragma unroll
-    for (int l = 0; l < SP_MAX_RANK; ++l)
-        if (l < p.rank) f |= (uint64_t)(first || (x >> p.shift[l]) != 0) << (kField * l);
-    return f;
-}
 
 __device__ __forceinline__ uint64_t warp_incl_scan64(uint64_t v) {
 #pragma unroll
@@ -520,24 +517,51 @@ __device__ __forceinline__ uint64_t block_excl_scan64(uint64_t v, uint64_t* sums
     return incl - v + pre;
 }
 
+// Per tile of kCtTile sorted entries: how many of them open a node at each level (packed 12-bit
+// counters).  Same entry-to-lane layout and the same test as k_emit below: a warp reads 32
+// consecutive keys per round, "opens a node at level l" is (significant bits of key ^ previous key)
+// > shift[l], and a count is the population count of a ballot.
+template <int RANK>
 __global__ void __launch_bounds__(kCtThreads)
 k_count_flags(const uint64_t* __restrict__ keys, int64_t n, LevelPlan p, uint64_t* __restrict__ tilesum) {
-    __shared__ uint64_t sums[16];
-    const int64_t e0 = (int64_t)blockIdx.x * kCtTile + (int64_t)threadIdx.x * kCtIpt;
-    uint64_t kprev = (e0 > 0 && e0 <= n) ? keys[e0 - 1] : 0;
-    uint64_t local = 0;
+    __shared__ uint32_t wtot[kCtThreads / 32][SP_MAX_RANK];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t chunk = (int64_t)blockIdx.x * kCtTile + (int64_t)w * (32 * kCtIpt);
+    uint64_t k[kCtIpt];
 #pragma unroll
     for (int i = 0; i < kCtIpt; ++i) {
-        int64_t e = e0 + i;
-        if (e < n) {
-            uint64_t k = keys[e];
-            local += level_flags(k, kprev, e == 0, p);
-            kprev = k;
-        }
+        const int64_t e = chunk + i * 32 + lane;
+        k[i] = e < n ? keys[e] : 0;
     }
-    uint64_t tot;
-    block_excl_scan64(local, sums, &tot);
-    if (threadIdx.x == 0) tilesum[blockIdx.x] = tot;
+    const uint64_t kbefore = (chunk > 0 && chunk <= n) ? keys[chunk - 1] : 0;
+    uint32_t tot[RANK];
+#pragma unroll
+    for (int l = 0; l < RANK; ++l) tot[l] = 0;
+#pragma unroll
+    for (int i = 0; i < kCtIpt; ++i) {
+        const int64_t e = chunk + i * 32 + lane;
+        const uint64_t up = __shfl_up_sync(0xffffffffu, k[i], 1);
+        const uint64_t wrap = i > 0 ? __shfl_sync(0xffffffffu, k[i > 0 ? i - 1 : 0], 31) : kbefore;
+        const uint64_t x = k[i] ^ (lane ? up : wrap);
+        const int hb = e >= n ? 0 : (e == 0 ? 64 : 64 - __clzll((long long)x));
+#pragma unroll
+        for (int l = 0; l < RANK; ++l) tot[l] += (uint32_t)__popc(__ballot_sync(0xffffffffu, hb > p.shift[l]));
+    }
+    if (lane == 0) {
+#pragma unroll
+        for (int l = 0; l < RANK; ++l) wtot[w][l] = tot[l];
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint64_t packed = 0;
+#pragma unroll
+        for (int l = 0; l < RANK; ++l) {
+            uint32_t c = 0;
+            for (int ww = 0; ww < kCtThreads / 32; ++ww) c += wtot[ww][l];
+            packed |= (uint64_t)c << (kField * l);
+        }
+        tilesum[blockIdx.x] = packed;
+    }
 }
 
 static_assert(kField * SP_MAX_RANK <= 64 && (1 << kField) > kCtTile, "packed per-tile counters");
@@ -564,8 +588,9 @@ k_scan_tiles(const uint64_t* __restrict__ tilesum, int64_t ntiles, int rank, int
 
 struct EmitArgs {
     const uint64_t* keys;
-    const uint32_t* idx;
-    const double* vals_in;
+    const uint32_t* idx;        // sorted position -> input entry (when the index rode in the key), else null
+    const double* vals_in;      // values in input order (read through idx)
+    const double* vals_sorted;  // values in sorted order (when they travelled with the keys), else null
     int64_t n;
     LevelPlan plan;
     const int64_t* tileprefix;
@@ -584,85 +609,124 @@ struct EmitArgs {
 #else
 #define SP_EMIT_BOUNDS __launch_bounds__(kCtThreads)
 #endif
+// Writes crd, first-child pos and values of one tile (the tiles of k_count_flags).  A warp owns 256
+// consecutive sorted entries and reads them 32 at a time, so every load and - node ids being
+// consecutive along the entries - every store of a warp instruction falls on consecutive addresses.
+// "Entry e opens a node at level l" is a comparison of the number of significant bits of
+// key[e] ^ key[e-1] with the level's shift, so a node id is a ballot and a population count: first
+// the warps total their flags per level, then (the totals exchanged through shared memory) each entry
+// gets its ids from the same ballots and walks its levels on its own.
+// W32: positions and coordinates are stored as 32-bit words (plain stores instead of a width switch).
+template <int RANK, bool W32>
 __global__ void SP_EMIT_BOUNDS k_emit(EmitArgs a) {
-    __shared__ uint64_t sums[16];
+    __shared__ uint32_t wtot[kCtThreads / 32][SP_MAX_RANK];
     const LevelPlan& p = a.plan;
-    const int64_t e0 = (int64_t)blockIdx.x * kCtTile + (int64_t)threadIdx.x * kCtIpt;
-    uint64_t k[kCtIpt], f[kCtIpt];
-    uint64_t kprev = (e0 > 0 && e0 <= a.n) ? a.keys[e0 - 1] : 0;
-    uint64_t local = 0;
-    {
-        uint64_t kp = kprev;
-#pragma unroll
-        for (int i = 0; i < kCtIpt; ++i) {
-            int64_t e = e0 + i;
-            k[i] = 0; f[i] = 0;
-            if (e < a.n) {
-                k[i] = a.keys[e];
-                f[i] = level_flags(k[i], kp, e == 0, p);
-                local += f[i];
-                kp = k[i];
-            }
-        }
-    }
-    uint64_t tot;
-    uint64_t ex = block_excl_scan64(local, sums, &tot);
-    int64_t incl[SP_MAX_RANK];
-#pragma unroll
-    for (int l = 0; l < SP_MAX_RANK; ++l)
-        incl[l] = l < p.rank ? a.tileprefix[(int64_t)l * a.ntiles + blockIdx.x] + (int64_t)((ex >> (kField * l)) & kFieldMask) : 0;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t chunk = (int64_t)blockIdx.x * kCtTile + (int64_t)w * (32 * kCtIpt);
+    const uint32_t le_mask = 0xffffffffu >> (31 - lane);          // lanes up to and including this one
 
-    // values of this thread's entries, gathered before the (sequential) level walk needs them
-    uint32_t id[kCtIpt];
-    double vin[kCtIpt];
-#pragma unroll
-    for (int i = 0; i < kCtIpt; ++i) id[i] = (e0 + i < a.n) ? a.idx[e0 + i] : 0u;
-#pragma unroll
-    for (int i = 0; i < kCtIpt; ++i) vin[i] = a.vals_in[(e0 + i < a.n) ? id[i] : 0u];
-    const bool next_same = (e0 + kCtIpt < a.n) && a.keys[e0 + kCtIpt] == k[kCtIpt - 1];
-
-    uint64_t kp = kprev;
+    uint64_t k[kCtIpt];
 #pragma unroll
     for (int i = 0; i < kCtIpt; ++i) {
-        int64_t e = e0 + i;
-        if (e >= a.n) break;
+        const int64_t e = chunk + i * 32 + lane;
+        k[i] = e < a.n ? a.keys[e] : 0;
+    }
+    const uint64_t kbefore = (chunk > 0 && chunk <= a.n) ? a.keys[chunk - 1] : 0;   // uniform per warp
+    // key of the entry before entry (i, lane)
+    auto prev_key = [&](int i) -> uint64_t {
+        const uint64_t up = __shfl_up_sync(0xffffffffu, k[i], 1);
+        const uint64_t wrap = i > 0 ? __shfl_sync(0xffffffffu, k[i > 0 ? i - 1 : 0], 31) : kbefore;
+        return lane ? up : wrap;
+    };
+    // significant bits of key ^ previous key (64 for the very first entry, 0 past the end): the entry
+    // opens a node at level l exactly when this exceeds shift[l]
+    int hb[kCtIpt];
+    uint32_t tot[RANK];
+#pragma unroll
+    for (int l = 0; l < RANK; ++l) tot[l] = 0;
+#pragma unroll
+    for (int i = 0; i < kCtIpt; ++i) {
+        const int64_t e = chunk + i * 32 + lane;
+        const uint64_t x = k[i] ^ prev_key(i);
+        hb[i] = e >= a.n ? 0 : (e == 0 ? 64 : 64 - __clzll((long long)x));
+#pragma unroll
+        for (int l = 0; l < RANK; ++l) tot[l] += (uint32_t)__popc(__ballot_sync(0xffffffffu, hb[i] > p.shift[l]));
+    }
+    if (lane == 0) {
+#pragma unroll
+        for (int l = 0; l < RANK; ++l) wtot[w][l] = tot[l];
+    }
+
+    // this thread's values, requested before the barrier
+    double vin[kCtIpt];
+    if (a.vals_sorted) {
+#pragma unroll
+        for (int i = 0; i < kCtIpt; ++i) { const int64_t e = chunk + i * 32 + lane; vin[i] = e < a.n ? a.vals_sorted[e] : 0.0; }
+    } else {
+        uint32_t id[kCtIpt];
+#pragma unroll
+        for (int i = 0; i < kCtIpt; ++i) { const int64_t e = chunk + i * 32 + lane; id[i] = e < a.n ? a.idx[e] : 0u; }
+#pragma unroll
+        for (int i = 0; i < kCtIpt; ++i) vin[i] = a.vals_in[id[i]];
+    }
+    __syncthreads();
+
+    int64_t run[RANK];                            // flagged entries at level l before this warp's round
+#pragma unroll
+    for (int l = 0; l < RANK; ++l) {
+        int64_t r = a.tileprefix[(int64_t)l * a.ntiles + blockIdx.x];
+        for (int ww = 0; ww < w; ++ww) r += wtot[ww][l];
+        run[l] = r;
+    }
+    const uint64_t knext = (chunk + 32 * kCtIpt < a.n) ? a.keys[chunk + 32 * kCtIpt] : ~0ull;   // uniform per warp
+#pragma unroll
+    for (int i = 0; i < kCtIpt; ++i) {
+        const int64_t e = chunk + i * 32 + lane;
+        const uint64_t kp = prev_key(i);
+        // does the entry after this one repeat its coordinates?  (its last-level flag is clear)
+        int hb_next = __shfl_down_sync(0xffffffffu, hb[i], 1);
+        const int hb_wrap = __shfl_sync(0xffffffffu, hb[i + 1 < kCtIpt ? i + 1 : i], 0);
+        if (lane == 31) hb_next = i + 1 < kCtIpt ? hb_wrap : ((e + 1 < a.n && knext == k[i]) ? 0 : 64);
         int64_t ppos = 0, pprev = 0;
         bool full = false;
 #pragma unroll
-        for (int l = 0; l < SP_MAX_RANK; ++l) {
-            if (l >= p.rank) continue;
+        for (int l = 0; l < RANK; ++l) {
+            const bool fl = hb[i] > p.shift[l];
+            const uint32_t m = __ballot_sync(0xffffffffu, fl);
+            const int64_t incl = run[l] + __popc(m & le_mask);
+            run[l] += __popc(m);
+            if (e >= a.n) continue;
             const uint64_t mask = p.bits[l] >= 64 ? ~0ull : ((1ull << p.bits[l]) - 1);
             const int64_t c = (int64_t)((k[i] >> p.shift[l]) & mask);
-            const int64_t cp = (int64_t)((kp >> p.shift[l]) & mask);
-            const bool fl = (f[i] >> (kField * l)) & 1;
-            incl[l] += fl;
-            if (l == p.rank - 1) full = fl;
+            if (l == RANK - 1) full = fl;
             if (p.lt[l] == SP_DENSE) {
+                const int64_t cp = (int64_t)((kp >> p.shift[l]) & mask);
                 ppos = ppos * p.sz[l] + c;
                 pprev = pprev * p.sz[l] + cp;
             } else {
-                const int64_t nid = incl[l] - 1;
+                const int64_t nid = incl - 1;
                 if (fl) {
-                    sp_store_uint(a.crd[l], nid, (uint64_t)c, a.crdBits);
-                    if (e == 0 || pprev != ppos) sp_store_uint(a.pos[l], ppos, (uint64_t)nid, a.posBits);
+                    if (W32) static_cast<uint32_t*>(a.crd[l])[nid] = (uint32_t)c;
+                    else sp_store_uint(a.crd[l], nid, (uint64_t)c, a.crdBits);
+                    if (e == 0 || pprev != ppos) {
+                        if (W32) static_cast<uint32_t*>(a.pos[l])[ppos] = (uint32_t)nid;
+                        else sp_store_uint(a.pos[l], ppos, (uint64_t)nid, a.posBits);
+                    }
                 }
                 pprev = nid - (fl ? 1 : 0);
                 ppos = nid;
             }
         }
+        if (e >= a.n) continue;
         if (full) {
-            // the entry after this one repeats the coordinates only when its "new position" flag is clear
-            const bool dup = (i + 1 < kCtIpt) ? (e + 1 < a.n && !((f[(i + 1) % kCtIpt] >> (kField * (p.rank - 1))) & 1))
-                                              : next_same;
             double s = vin[i];
-            if (dup)
-                for (int64_t g = e + 1; g < a.n && a.keys[g] == k[i]; ++g) s += a.vals_in[a.idx[g]];
+            if (e + 1 < a.n && !(hb_next > p.shift[RANK - 1]))   // rare: the run of equal coordinates is summed by its first entry
+                for (int64_t g = e + 1; g < a.n && a.keys[g] == k[i]; ++g) s += a.vals_sorted ? a.vals_sorted[g] : a.vals_in[a.idx[g]];
             a.val[ppos] = s;
             if (a.seg_out) a.seg_out[ppos] = (uint32_t)(k[i] >> p.shift[0]);
         } else if (a.flags & SP_DUP_ERROR) {
             atomicOr(a.err, kErrDup);
         }
-        kp = k[i];
     }
 }
 
@@ -860,20 +924,25 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
     const int64_t n = nnz;
     int64_t counts[SP_MAX_RANK] = {};
     uint64_t* keys = nullptr;
-    uint32_t* idx = nullptr;
+    uint32_t* idx = nullptr;            // sorted position -> input entry (index-in-key sorts)
+    const double* vals_sorted = nullptr;   // or the values in sorted order (value-beside-key sorts)
     int64_t* tileprefix = nullptr;
     int* d_err = nullptr;
     int64_t ct_tiles = 0;
 
     if (n > 0) {
         uint64_t* kbuf[2] = {ws.get<uint64_t>((size_t)n), ws.get<uint64_t>((size_t)n)};
-        uint32_t* ibuf[2] = {ws.get<uint32_t>((size_t)n), ws.get<uint32_t>((size_t)n)};
         d_err = ws.get<int>(1);
         const int npasses = (total_bits + kMaxDigitBits - 1) / kMaxDigitBits;
-        // the entry index rides inside the key when both fit in 64 bits
+        // the entry index rides inside the key when both fit in 64 bits; otherwise the values travel
+        // beside the keys (one array per side of the ping-pong; the first pass reads the input's)
         int idx_bits = 0;
         while (((int64_t)1 << idx_bits) < n) ++idx_bits;
         const bool fused = npasses > 0 && idx_bits > 0 && total_bits + idx_bits <= 64;
+        uint64_t* pbuf[2] = {nullptr, nullptr};
+        uint32_t* isorted = nullptr;
+        if (fused) isorted = ws.get<uint32_t>((size_t)n);
+        else if (npasses > 0) { pbuf[0] = ws.get<uint64_t>((size_t)n); pbuf[1] = ws.get<uint64_t>((size_t)n); }
         const int64_t stiles = sp_ceil_div(n, fused ? SortShape<false>::kTile : SortShape<true>::kTile);
         uint32_t* tilehist = ws.get<uint32_t>((size_t)stiles << kMaxDigitBits);
         uint32_t* digit_total = ws.get<uint32_t>((size_t)1 << kMaxDigitBits);
@@ -898,7 +967,7 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         const int shift0 = npasses ? shifts[0] : 0;
         const uint32_t mask0 = npasses ? (1u << widths[0]) - 1u : 0u;
 #define SP_BUILD_KEYS(CT, PAY)                                                                                       \
-    k_build_keys<CT, PAY><<<(unsigned)stiles, kSortThreads, 0, stream>>>(lc, n, plan, kbuf[0], ibuf[0], fused ? idx_bits : 0, \
+    k_build_keys<CT, PAY><<<(unsigned)stiles, kSortThreads, 0, stream>>>(lc, n, plan, kbuf[0], fused ? idx_bits : 0,         \
                                                                         d_err, shift0, mask0, tilehist, stiles)
         if (coo_coord_bits == 32) { if (fused) SP_BUILD_KEYS(int32_t, false); else SP_BUILD_KEYS(int32_t, true); }
         else { if (fused) SP_BUILD_KEYS(int64_t, false); else SP_BUILD_KEYS(int64_t, true); }
@@ -913,7 +982,8 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
             sp_status ps_st = SP_ERR_UNSUPPORTED;
 #define SP_SORT_PASS(B)                                                                                             \
     case B:                                                                                                         \
-        ps_st = sort_pass<B>(kbuf[cur], ibuf[cur], kbuf[cur ^ 1], ibuf[cur ^ 1], n, shifts[ps], tilehist, stiles,    \
+        ps_st = sort_pass<B>(kbuf[cur], ps == 0 ? reinterpret_cast<const uint64_t*>(coo_vals) : pbuf[cur],          \
+                             kbuf[cur ^ 1], pbuf[cur ^ 1], isorted, n, shifts[ps], tilehist, stiles,                 \
                              digit_total, chunk_tot, fused, split, ps == 0, stream, timer);                          \
         break;
             switch (widths[ps]) {
@@ -926,9 +996,16 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         }
         npasses_done = npasses;
         keys = kbuf[cur];
-        idx = ibuf[cur];
+        if (fused) idx = isorted;
+        else vals_sorted = npasses > 0 ? reinterpret_cast<const double*>(pbuf[cur]) : coo_vals;   // no pass: one cell
 
-        k_count_flags<<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum);
+        switch (rank) {
+            case 1: k_count_flags<1><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum); break;
+            case 2: k_count_flags<2><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum); break;
+            case 3: k_count_flags<3><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum); break;
+            case 4: k_count_flags<4><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum); break;
+            default: k_count_flags<5><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum); break;
+        }
         k_scan_tiles<<<rank, 512, 0, stream>>>(tilesum, ct_tiles, rank, tileprefix, d_counts);
         SP_LAUNCH_CHECK();
         timer.mark(kPhCount);
@@ -990,7 +1067,7 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
     }
     if (n > 0) {
         EmitArgs a;
-        a.keys = keys; a.idx = idx; a.vals_in = coo_vals; a.n = n; a.plan = plan;
+        a.keys = keys; a.idx = idx; a.vals_in = coo_vals; a.vals_sorted = vals_sorted; a.n = n; a.plan = plan;
         a.tileprefix = tileprefix; a.ntiles = ct_tiles;
         for (int l = 0; l < SP_MAX_RANK; ++l) { a.pos[l] = t->pos[l]; a.crd[l] = t->crd[l]; }
         a.val = t->val; a.posBits = posBits; a.crdBits = crdBits; a.flags = flags; a.err = d_err;
@@ -1004,7 +1081,14 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
             a.seg_out = reinterpret_cast<uint32_t*>(sg.aux);
             t->parts[(uint64_t)SP_PART_SEGIDS << 56] = sg;
         }
-        k_emit<<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);
+        const bool w32 = posBits == 32 && crdBits == 32;
+#define SP_EMIT(R)                                                                              \
+    case R:                                                                                     \
+        if (w32) k_emit<R, true><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);             \
+        else k_emit<R, false><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);                \
+        break;
+        switch (rank) { SP_EMIT(1) SP_EMIT(2) SP_EMIT(3) SP_EMIT(4) SP_EMIT(5) }
+#undef SP_EMIT
         sp_count_launches(1);
         for (int l = 0; l < rank; ++l) {
             if (plan.lt[l] != SP_COMPRESSED) continue;
