@@ -617,7 +617,9 @@ struct EmitArgs {
 // the warps total their flags per level, then (the totals exchanged through shared memory) each entry
 // gets its ids from the same ballots and walks its levels on its own.
 // W32: positions and coordinates are stored as 32-bit words (plain stores instead of a width switch).
-template <int RANK, bool W32>
+// ALLC: every level is compressed, so a node's parent position is the parent's node id and "my parent
+// is new" is the previous level's flag: no linearised positions, no look at the previous key.
+template <int RANK, bool W32, bool ALLC>
 __global__ void SP_EMIT_BOUNDS k_emit(EmitArgs a) {
     __shared__ uint32_t wtot[kCtThreads / 32][SP_MAX_RANK];
     const LevelPlan& p = a.plan;
@@ -671,10 +673,10 @@ __global__ void SP_EMIT_BOUNDS k_emit(EmitArgs a) {
     }
     __syncthreads();
 
-    int64_t run[RANK];                            // flagged entries at level l before this warp's round
+    uint32_t run[RANK];                           // flagged entries at level l before this warp's round (< nnz < 2^32)
 #pragma unroll
     for (int l = 0; l < RANK; ++l) {
-        int64_t r = a.tileprefix[(int64_t)l * a.ntiles + blockIdx.x];
+        uint32_t r = (uint32_t)a.tileprefix[(int64_t)l * a.ntiles + blockIdx.x];
         for (int ww = 0; ww < w; ++ww) r += wtot[ww][l];
         run[l] = r;
     }
@@ -682,39 +684,65 @@ __global__ void SP_EMIT_BOUNDS k_emit(EmitArgs a) {
 #pragma unroll
     for (int i = 0; i < kCtIpt; ++i) {
         const int64_t e = chunk + i * 32 + lane;
-        const uint64_t kp = prev_key(i);
         // does the entry after this one repeat its coordinates?  (its last-level flag is clear)
         int hb_next = __shfl_down_sync(0xffffffffu, hb[i], 1);
         const int hb_wrap = __shfl_sync(0xffffffffu, hb[i + 1 < kCtIpt ? i + 1 : i], 0);
         if (lane == 31) hb_next = i + 1 < kCtIpt ? hb_wrap : ((e + 1 < a.n && knext == k[i]) ? 0 : 64);
-        int64_t ppos = 0, pprev = 0;
+        int64_t ppos = 0;
         bool full = false;
+        if (ALLC) {
+            uint32_t parent = 0;
+            bool parent_new = e == 0;
 #pragma unroll
-        for (int l = 0; l < RANK; ++l) {
-            const bool fl = hb[i] > p.shift[l];
-            const uint32_t m = __ballot_sync(0xffffffffu, fl);
-            const int64_t incl = run[l] + __popc(m & le_mask);
-            run[l] += __popc(m);
-            if (e >= a.n) continue;
-            const uint64_t mask = p.bits[l] >= 64 ? ~0ull : ((1ull << p.bits[l]) - 1);
-            const int64_t c = (int64_t)((k[i] >> p.shift[l]) & mask);
-            if (l == RANK - 1) full = fl;
-            if (p.lt[l] == SP_DENSE) {
-                const int64_t cp = (int64_t)((kp >> p.shift[l]) & mask);
-                ppos = ppos * p.sz[l] + c;
-                pprev = pprev * p.sz[l] + cp;
-            } else {
-                const int64_t nid = incl - 1;
-                if (fl) {
+            for (int l = 0; l < RANK; ++l) {
+                const bool fl = hb[i] > p.shift[l];
+                const uint32_t m = __ballot_sync(0xffffffffu, fl);
+                const uint32_t nid = run[l] + (uint32_t)__popc(m & le_mask) - 1u;
+                run[l] += (uint32_t)__popc(m);
+                if (fl) {                              // never set past the end
+                    const uint64_t c = (k[i] >> p.shift[l]) & (((uint64_t)1 << p.bits[l]) - 1);   // bits[l] <= 63
                     if (W32) static_cast<uint32_t*>(a.crd[l])[nid] = (uint32_t)c;
-                    else sp_store_uint(a.crd[l], nid, (uint64_t)c, a.crdBits);
-                    if (e == 0 || pprev != ppos) {
-                        if (W32) static_cast<uint32_t*>(a.pos[l])[ppos] = (uint32_t)nid;
-                        else sp_store_uint(a.pos[l], ppos, (uint64_t)nid, a.posBits);
+                    else sp_store_uint(a.crd[l], nid, c, a.crdBits);
+                    if (parent_new) {
+                        if (W32) static_cast<uint32_t*>(a.pos[l])[parent] = nid;
+                        else sp_store_uint(a.pos[l], parent, (uint64_t)nid, a.posBits);
                     }
                 }
-                pprev = nid - (fl ? 1 : 0);
-                ppos = nid;
+                parent = nid;
+                parent_new = fl;
+            }
+            full = parent_new;
+            ppos = parent;
+        } else {
+            const uint64_t kp = prev_key(i);
+            int64_t pprev = 0;
+#pragma unroll
+            for (int l = 0; l < RANK; ++l) {
+                const bool fl = hb[i] > p.shift[l];
+                const uint32_t m = __ballot_sync(0xffffffffu, fl);
+                const int64_t incl = (int64_t)(run[l] + (uint32_t)__popc(m & le_mask));
+                run[l] += (uint32_t)__popc(m);
+                if (e >= a.n) continue;
+                const uint64_t mask = p.bits[l] >= 64 ? ~0ull : ((1ull << p.bits[l]) - 1);
+                const int64_t c = (int64_t)((k[i] >> p.shift[l]) & mask);
+                if (l == RANK - 1) full = fl;
+                if (p.lt[l] == SP_DENSE) {
+                    const int64_t cp = (int64_t)((kp >> p.shift[l]) & mask);
+                    ppos = ppos * p.sz[l] + c;
+                    pprev = pprev * p.sz[l] + cp;
+                } else {
+                    const int64_t nid = incl - 1;
+                    if (fl) {
+                        if (W32) static_cast<uint32_t*>(a.crd[l])[nid] = (uint32_t)c;
+                        else sp_store_uint(a.crd[l], nid, (uint64_t)c, a.crdBits);
+                        if (e == 0 || pprev != ppos) {
+                            if (W32) static_cast<uint32_t*>(a.pos[l])[ppos] = (uint32_t)nid;
+                            else sp_store_uint(a.pos[l], ppos, (uint64_t)nid, a.posBits);
+                        }
+                    }
+                    pprev = nid - (fl ? 1 : 0);
+                    ppos = nid;
+                }
             }
         }
         if (e >= a.n) continue;
@@ -1082,10 +1110,17 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
             t->parts[(uint64_t)SP_PART_SEGIDS << 56] = sg;
         }
         const bool w32 = posBits == 32 && crdBits == 32;
+        bool allc = true;
+        for (int l = 0; l < rank; ++l) allc = allc && plan.lt[l] == SP_COMPRESSED;
 #define SP_EMIT(R)                                                                              \
     case R:                                                                                     \
-        if (w32) k_emit<R, true><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);             \
-        else k_emit<R, false><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);                \
+        if (allc) {                                                                             \
+            if (w32) k_emit<R, true, true><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);   \
+            else k_emit<R, false, true><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);      \
+        } else {                                                                                \
+            if (w32) k_emit<R, true, false><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);  \
+            else k_emit<R, false, false><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);     \
+        }                                                                                       \
         break;
         switch (rank) { SP_EMIT(1) SP_EMIT(2) SP_EMIT(3) SP_EMIT(4) SP_EMIT(5) }
 #undef SP_EMIT
