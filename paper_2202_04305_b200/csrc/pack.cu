@@ -81,11 +81,17 @@ constexpr int kSortThreads = 256;
 // (six scatter passes over 20,000,000 entries: 0.78 ms against 0.87 ms with 16 keys and three tiles);
 // with the index inside the key (8-byte words) 16 keys per thread and three tiles per SM are
 // (5,000,000 entries: pack 0.48 ms against 0.50 ms).  Every kernel of one sort uses the same shape.
+#ifndef SP_SORT_PAY_IPT
+#define SP_SORT_PAY_IPT 8
+#endif
+#ifndef SP_SORT_PAY_BLOCKS
+#define SP_SORT_PAY_BLOCKS 4
+#endif
 template <bool PAY>
 struct SortShape {
-    static constexpr int kIpt = PAY ? 8 : 16;
+    static constexpr int kIpt = PAY ? SP_SORT_PAY_IPT : 16;
     static constexpr int kTile = kSortThreads * kIpt;
-    static constexpr int kMinBlocks = PAY ? 4 : 3;
+    static constexpr int kMinBlocks = PAY ? SP_SORT_PAY_BLOCKS : 3;
 };
 constexpr int kSortWarps = kSortThreads / 32;
 constexpr int kMaxRadix = 256;
@@ -356,9 +362,13 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint64_t* __restric
     for (int i = 0; i < kSortIpt; ++i) {             // all key loads first
         const int li = w * (32 * kSortIpt) + i * 32 + lane;
         key[i] = li < tile_n ? keys_in[base + li] : 0;
+#ifdef SP_SORT_PAY_EARLY
+        if (PAY) pay[i] = li < tile_n ? pay_in[base + li] : 0;
+#endif
     }
     if (tile_n == kSortTile) rank_rounds<BITS, BITS, kSortIpt>(key, shift, w, lane, tile_n, mycnt, rank);
     else rank_rounds<BITS, BITS + 1, kSortIpt>(key, shift, w, lane, tile_n, mycnt, rank);
+#ifndef SP_SORT_PAY_EARLY
     if (PAY) {
         // the payloads are not needed before the exchange: requested here, they arrive during the
         // digit scans below without holding registers through the ranking
@@ -368,6 +378,7 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint64_t* __restric
             pay[i] = li < tile_n ? pay_in[base + li] : 0;
         }
     }
+#endif
     __syncthreads();
 
     // per digit: exclusive scan over warps; then exclusive scan over digits (each thread owns
