@@ -256,7 +256,8 @@ constexpr int kBBox = kTK * 8;                 // doubles in one box of B
 constexpr int kStageDoubles = (kTK / 4) * kABox + 4 * kBBox;
 constexpr uint32_t kStageBytes = kStageDoubles * sizeof(double);
 constexpr size_t kTmaSmem = (size_t)kTStages * kStageBytes + kTStages * sizeof(uint64_t) + 128;
-constexpr int kWaitLimit = 1 << 22;            // polls of one mbarrier before the block gives up
+constexpr uint32_t kWaitPollNs = 2000;         // one poll of an mbarrier may sleep this long ...
+constexpr int kWaitLimit = 1 << 19;            // ... and a block gives up after this many polls: about a second
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -270,9 +271,9 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity), "r"(kWaitPollNs) : "memory");
     return ok != 0;
 }
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
