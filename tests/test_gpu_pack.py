@@ -97,7 +97,7 @@ def test_duplicates_zeros_and_flags(oracle):
     for lt, od in [((0, 1), (0, 1)), ((1, 1), (1, 0)), ((1, 0), (0, 1))]:
         t, ref = _pack_both(oracle, dup, lt, od)
         assert_storage_equal(t, ref)          # same summation order => same bits
-    # the same with keys too wide to carry the entry index inside them (the index travels as a payload then)
+    # the same with keys too wide to carry the entry index inside them (the value travels beside the key then)
     wide = I.uniform_tensor((1 << 20, 1 << 20, 1 << 20), 3000, seed=9)
     wc = [np.concatenate([c, c[:400], c[100:300]]) for c in wide.coords]
     wv = np.concatenate([wide.vals, I.uniform_pm1(8, 71, 600)])
@@ -110,6 +110,29 @@ def test_duplicates_zeros_and_flags(oracle):
     assert e.value.code == 5
     c, v = to_dev(coo)
     b.sp_pack(coo.dims, c, v, (0, 1), None, 32, 32, b.DUP_ERROR)   # duplicate-free input passes
+
+
+@pytest.mark.parametrize("wide", [False, True])
+def test_duplicate_runs_across_warp_and_tile_boundaries(oracle, wide):
+    """Runs of equal coordinates longer than a warp's round (32), a warp's share (256) and a tile (2048),
+    placed so that they straddle those boundaries in sorted order; summed in input order, so the bits
+    must match the oracle's.  wide: keys that cannot hold the entry index (values travel with the keys)."""
+    dims = (1 << 20, 1 << 20, 1 << 20) if wide else (64, 64, 64)
+    base = I.uniform_tensor(dims, 3000, seed=41)
+    reps = {5: 40, 700: 300, 701: 31, 1500: 2500, 2999: 270}      # entry of the base list -> copies of it
+    cols = [[c] for c in base.coords]
+    for e, r in reps.items():
+        for d in range(3):
+            cols[d].append(np.full(r, base.coords[d][e]))
+    coords = [np.concatenate(c) for c in cols]
+    n = coords[0].size
+    vals = I.uniform_pm1(41, 5, n)
+    perm = np.argsort(I.uniform_pm1(41, 6, n), kind="stable")       # a seeded shuffle of the input order
+    coo = I.Coo(dims, [c[perm] for c in coords], vals[perm])
+    for lt, od in [((1, 1, 1), (0, 1, 2)), ((0, 1, 1), (2, 0, 1))] if not wide else [((1, 1, 1), (0, 1, 2)), ((1, 1, 1), (2, 1, 0))]:
+        t, ref = _pack_both(oracle, coo, lt, od)
+        assert_storage_equal(t, ref)
+        assert t.nval == 3000 if lt == (1, 1, 1) else True
 
 
 def test_error_codes():
