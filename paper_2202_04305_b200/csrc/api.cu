@@ -72,11 +72,15 @@ sp_status sp_free(sp_tensor* t) {
     int prev = 0;
     cudaGetDevice(&prev);
     cudaSetDevice(t->device);
-    for (int l = 0; l < SP_MAX_RANK; ++l) {
-        sp_dev_free(t->pos[l], nullptr);
-        sp_dev_free(t->crd[l], nullptr);
+    if (t->block) {
+        sp_dev_free(t->block, nullptr);
+    } else {
+        for (int l = 0; l < SP_MAX_RANK; ++l) {
+            sp_dev_free(t->pos[l], nullptr);
+            sp_dev_free(t->crd[l], nullptr);
+        }
+        if (t->owns_val) sp_dev_free(t->val, nullptr);
     }
-    if (t->owns_val) sp_dev_free(t->val, nullptr);
     if (t->wide) sp_free(t->wide);
     for (auto& kv : t->parts) {
         sp_dev_free(kv.second.row, nullptr);

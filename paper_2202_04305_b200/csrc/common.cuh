@@ -48,6 +48,7 @@ struct sp_tensor {
     int64_t max_seg = -1;      // longest segment of the last level (entries under one parent); -1 = not measured yet
     sp_tensor* wide = nullptr;
     bool owns_val = true;
+    void* block = nullptr;   // when set: pos[], crd[] and val are pieces of this one allocation
 };
 
 // SP_ERR_INVALID_ARG unless the handle's arrays live on the current device.
@@ -70,12 +71,35 @@ struct sp_workspace {
     cudaStream_t stream;
     std::vector<void*> ptrs;
     bool failed = false;
+    char* pool = nullptr;          // what is left of a reserve()d block
+    size_t pool_left = 0;
     explicit sp_workspace(cudaStream_t s) : stream(s) {}
     ~sp_workspace() {
         for (void* p : ptrs) sp_dev_free(p, stream);
     }
+    static size_t padded(size_t bytes) { return (bytes + 255) & ~(size_t)255; }
+    template <typename T>
+    static size_t bytes_for(size_t count) { return padded((count ? count : 1) * sizeof(T)); }
+    // One trip to the allocator for buffers whose sizes are known up front (an allocator call can cost
+    // microseconds of host time while the GPU idles): the get()s that follow carve 256-byte aligned
+    // pieces out of this block and go to the allocator themselves only once it is used up.
+    void reserve(size_t bytes) {
+        if (bytes == 0) return;
+        void* p = sp_dev_alloc(bytes, stream);
+        if (!p) { failed = true; return; }
+        ptrs.push_back(p);
+        pool = static_cast<char*>(p);
+        pool_left = bytes;
+    }
     template <typename T>
     T* get(size_t count) {
+        const size_t need = bytes_for<T>(count);
+        if (pool && need <= pool_left) {
+            T* r = reinterpret_cast<T*>(pool);
+            pool += need;
+            pool_left -= need;
+            return r;
+        }
         void* p = sp_dev_alloc((count ? count : 1) * sizeof(T), stream);
         if (!p) { failed = true; return nullptr; }
         ptrs.push_back(p);

@@ -411,7 +411,7 @@ TmaHost& tma_host() {
             return;
         }
         void* word = nullptr;
-        if (cudaHostAlloc(&word, sizeof(int), cudaHostAllocMapped) != cudaSuccess) { (void)cudaGetLastError(); return; }
+        if (cudaHostAlloc(&word, sizeof(int), cudaHostAllocMapped | cudaHostAllocPortable) != cudaSuccess) { (void)cudaGetLastError(); return; }
         *static_cast<int*>(word) = 0;
         void* dev = nullptr;
         if (cudaHostGetDevicePointer(&dev, word, 0) != cudaSuccess) { (void)cudaGetLastError(); cudaFreeHost(word); return; }
@@ -466,16 +466,24 @@ sp_status spmm_dense_inner_tma(const sp_tensor* A, const void* outer, int64_t ns
         else SP_CUDA(cudaMemset2DAsync(C, (size_t)ldc * sizeof(double), 0, (size_t)N * sizeof(double), (size_t)m, stream));
     }
     dim3 grid((unsigned)rb, (unsigned)cb, (unsigned)ksplit);
-    static std::once_flag attr32, attr64;
-    if (A->crdBits == 32) {
-        std::call_once(attr32, [] { cudaFuncSetAttribute(k_spmm_dense_inner_tma<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaSmem); });
+    // the dynamic shared-memory limit is a per-device attribute of the function: raised once per device
+    static std::mutex attr_mutex;
+    static uint64_t attr_done[2] = {0, 0};          // [coordinate width], one bit per device
+    const int wi = A->crdBits == 32 ? 0 : 1;
+    {
+        std::lock_guard<std::mutex> lock(attr_mutex);
+        if (A->device < 0 || A->device >= 64 || !((attr_done[wi] >> A->device) & 1)) {
+            SP_CUDA(wi == 0 ? cudaFuncSetAttribute(k_spmm_dense_inner_tma<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaSmem)
+                            : cudaFuncSetAttribute(k_spmm_dense_inner_tma<uint64_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaSmem));
+            if (A->device >= 0 && A->device < 64) attr_done[wi] |= (uint64_t)1 << A->device;
+        }
+    }
+    if (wi == 0)
         k_spmm_dense_inner_tma<uint32_t><<<grid, kTThreads, kTmaSmem, stream>>>(map_a, map_b, static_cast<const uint32_t*>(outer), nslices,
                                                                                 inner, N, C, ldc, kchunk, h.gave_up_dev);
-    } else {
-        std::call_once(attr64, [] { cudaFuncSetAttribute(k_spmm_dense_inner_tma<uint64_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaSmem); });
+    else
         k_spmm_dense_inner_tma<uint64_t><<<grid, kTThreads, kTmaSmem, stream>>>(map_a, map_b, static_cast<const uint64_t*>(outer), nslices,
                                                                                 inner, N, C, ldc, kchunk, h.gave_up_dev);
-    }
     SP_LAUNCH_CHECK();
     sp_count_launches(1);
     return SP_OK;

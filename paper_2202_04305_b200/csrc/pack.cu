@@ -970,23 +970,31 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
     int64_t ct_tiles = 0;
 
     if (n > 0) {
-        uint64_t* kbuf[2] = {ws.get<uint64_t>((size_t)n), ws.get<uint64_t>((size_t)n)};
-        d_err = ws.get<int>(1);
         const int npasses = (total_bits + kMaxDigitBits - 1) / kMaxDigitBits;
         // the entry index rides inside the key when both fit in 64 bits; otherwise the values travel
         // beside the keys (one array per side of the ping-pong; the first pass reads the input's)
         int idx_bits = 0;
         while (((int64_t)1 << idx_bits) < n) ++idx_bits;
         const bool fused = npasses > 0 && idx_bits > 0 && total_bits + idx_bits <= 64;
+        const int64_t stiles = sp_ceil_div(n, fused ? SortShape<false>::kTile : SortShape<true>::kTile);
+        ct_tiles = sp_ceil_div(n, kCtTile);
+        const size_t nscan = (size_t)sp_ceil_div(stiles, kScanChunk) << kMaxDigitBits;
+        // every buffer of the pack in one allocation
+        ws.reserve(2 * sp_workspace::bytes_for<uint64_t>((size_t)n) +
+                   (fused ? sp_workspace::bytes_for<uint32_t>((size_t)n) : npasses > 0 ? 2 * sp_workspace::bytes_for<uint64_t>((size_t)n) : 0) +
+                   sp_workspace::bytes_for<int>(1) + sp_workspace::bytes_for<uint32_t>((size_t)stiles << kMaxDigitBits) +
+                   sp_workspace::bytes_for<uint32_t>((size_t)1 << kMaxDigitBits) + sp_workspace::bytes_for<uint32_t>(nscan) +
+                   sp_workspace::bytes_for<uint64_t>((size_t)ct_tiles) + sp_workspace::bytes_for<int64_t>((size_t)ct_tiles * SP_MAX_RANK) +
+                   sp_workspace::bytes_for<int64_t>(SP_MAX_RANK));
+        uint64_t* kbuf[2] = {ws.get<uint64_t>((size_t)n), ws.get<uint64_t>((size_t)n)};
+        d_err = ws.get<int>(1);
         uint64_t* pbuf[2] = {nullptr, nullptr};
         uint32_t* isorted = nullptr;
         if (fused) isorted = ws.get<uint32_t>((size_t)n);
         else if (npasses > 0) { pbuf[0] = ws.get<uint64_t>((size_t)n); pbuf[1] = ws.get<uint64_t>((size_t)n); }
-        const int64_t stiles = sp_ceil_div(n, fused ? SortShape<false>::kTile : SortShape<true>::kTile);
         uint32_t* tilehist = ws.get<uint32_t>((size_t)stiles << kMaxDigitBits);
         uint32_t* digit_total = ws.get<uint32_t>((size_t)1 << kMaxDigitBits);
-        uint32_t* chunk_tot = ws.get<uint32_t>((size_t)sp_ceil_div(stiles, kScanChunk) << kMaxDigitBits);
-        ct_tiles = sp_ceil_div(n, kCtTile);
+        uint32_t* chunk_tot = ws.get<uint32_t>(nscan);
         uint64_t* tilesum = ws.get<uint64_t>((size_t)ct_tiles);
         tileprefix = ws.get<int64_t>((size_t)ct_tiles * SP_MAX_RANK);
         int64_t* d_counts = ws.get<int64_t>(SP_MAX_RANK);
@@ -1079,16 +1087,33 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
             if ((uint64_t)counts[l] > max_pos) { st = SP_ERR_WIDTH_OVERFLOW; break; }
             t->npos[l] = parents + 1;
             t->ncrd[l] = counts[l];
-            t->pos[l] = sp_dev_alloc((size_t)t->npos[l] * pw, stream);
-            t->crd[l] = sp_dev_alloc((size_t)(counts[l] ? counts[l] : 1) * cw, stream);
-            if (!t->pos[l] || !t->crd[l]) { st = SP_ERR_ALLOC; break; }
             parents = counts[l];
         }
     }
     if (st == SP_OK) {
+        // one allocation holds every array of the handle (each piece 256-byte aligned): an allocator
+        // call costs host time during which the GPU, drained by the read-back above, has nothing to do
         t->nval = parents;
-        t->val = static_cast<double*>(sp_dev_alloc((size_t)(parents ? parents : 1) * sizeof(double), stream));
-        if (!t->val) st = SP_ERR_ALLOC;
+        size_t off_pos[SP_MAX_RANK] = {}, off_crd[SP_MAX_RANK] = {}, total = 0;
+        for (int l = 0; l < rank; ++l) {
+            if (plan.lt[l] != SP_COMPRESSED) continue;
+            off_pos[l] = total; total += sp_workspace::padded((size_t)t->npos[l] * pw);
+            off_crd[l] = total; total += sp_workspace::padded((size_t)(t->ncrd[l] ? t->ncrd[l] : 1) * cw);
+        }
+        const size_t off_val = total;
+        total += sp_workspace::padded((size_t)(parents ? parents : 1) * sizeof(double));
+        t->block = sp_dev_alloc(total, stream);
+        if (!t->block) {
+            st = SP_ERR_ALLOC;
+        } else {
+            char* base = static_cast<char*>(t->block);
+            for (int l = 0; l < rank; ++l) {
+                if (plan.lt[l] != SP_COMPRESSED) continue;
+                t->pos[l] = base + off_pos[l];
+                t->crd[l] = base + off_crd[l];
+            }
+            t->val = reinterpret_cast<double*>(base + off_val);
+        }
     }
     if (st != SP_OK) { sp_free(t); return st; }
 

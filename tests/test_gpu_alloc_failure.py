@@ -93,7 +93,7 @@ def test_pack_gives_everything_back(alloc, lt, od):
     coo = I.config3(seed=5, n=1 << 10, nnz=6000)
     coords, vals = to_dev(coo)
     pts = sweep(alloc, lambda: sp().sp_pack(coo.dims, coords, vals, lt, od))
-    assert pts >= 8          # keys, indices, histograms, tile sums, level arrays, values ...
+    assert pts >= 2          # the pack's workspace (one block), the handle's arrays (one block), scan scratch ...
     alloc.arm(0)
     sp().sp_pack(coo.dims, coords, vals, lt, od).free()     # and the next call works
 
@@ -101,10 +101,10 @@ def test_pack_gives_everything_back(alloc, lt, od):
 def test_pack_rank3_and_convert(alloc):
     t = I.config5(seed=5, dim=64, nnz=5000)
     coords, vals = to_dev(t)
-    assert sweep(alloc, lambda: sp().sp_pack(t.dims, coords, vals, (0, 1, 1))) >= 8
+    assert sweep(alloc, lambda: sp().sp_pack(t.dims, coords, vals, (0, 1, 1))) >= 2
     alloc.arm(0)
     T = sp().sp_pack(t.dims, coords, vals, (1, 1, 1))
-    assert sweep(alloc, lambda: sp().sp_convert(T, (0, 1, 1), (0, 2, 1))) >= 8
+    assert sweep(alloc, lambda: sp().sp_convert(T, (0, 1, 1), (0, 2, 1))) >= 3
     T.free()
 
 
