@@ -613,6 +613,8 @@ struct EmitArgs {
     int posBits, crdBits;
     unsigned flags;
     int* err;
+    int64_t last_pos[SP_MAX_RANK];   // index of the closing entry of pos[l] (its parents' count) ...
+    int64_t last_val[SP_MAX_RANK];   // ... and what goes there: the level's node count
 };
 
 #ifdef SP_LB_EMIT
@@ -644,6 +646,8 @@ __global__ void SP_EMIT_BOUNDS k_emit(EmitArgs a) {
         const int64_t e = chunk + i * 32 + lane;
         k[i] = e < a.n ? a.keys[e] : 0;
     }
+    if (blockIdx.x == 0 && threadIdx.x < RANK && p.lt[threadIdx.x] == SP_COMPRESSED)   // pos[l] ends with the node count
+        sp_store_uint(a.pos[threadIdx.x], a.last_pos[threadIdx.x], (uint64_t)a.last_val[threadIdx.x], a.posBits);
     const uint64_t kbefore = (chunk > 0 && chunk <= a.n) ? a.keys[chunk - 1] : 0;   // uniform per warp
     // key of the entry before entry (i, lane)
     auto prev_key = [&](int i) -> uint64_t {
@@ -768,8 +772,6 @@ __global__ void SP_EMIT_BOUNDS k_emit(EmitArgs a) {
         }
     }
 }
-
-__global__ void k_store_one(void* base, int64_t i, uint64_t v, int bits) { sp_store_uint(base, i, v, bits); }
 
 // --------------------------------------------- suffix-min fill of pos[] ---
 // a[i] <- min(a[i..L-1]).  Written as a forward scan over r = L-1-i.
@@ -1135,6 +1137,7 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         a.tileprefix = tileprefix; a.ntiles = ct_tiles;
         for (int l = 0; l < SP_MAX_RANK; ++l) { a.pos[l] = t->pos[l]; a.crd[l] = t->crd[l]; }
         a.val = t->val; a.posBits = posBits; a.crdBits = crdBits; a.flags = flags; a.err = d_err;
+        for (int l = 0; l < SP_MAX_RANK; ++l) { a.last_pos[l] = parents_at[l]; a.last_val[l] = counts[l]; }
         // Column-major matrices run SpMM as a flat loop over entries and need each entry's column:
         // it is in the sorted key anyway, so it is written here instead of being searched for later.
         a.seg_out = nullptr;
@@ -1163,8 +1166,6 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         sp_count_launches(1);
         for (int l = 0; l < rank; ++l) {
             if (plan.lt[l] != SP_COMPRESSED) continue;
-            k_store_one<<<1, 1, 0, stream>>>(t->pos[l], parents_at[l], (uint64_t)counts[l], posBits);
-            sp_count_launches(1);
             if (needs_fill[l]) {
                 sp_status s2 = posBits == 64   ? suffix_min_inplace<uint64_t>(t->pos[l], t->npos[l], stream)
                                : posBits == 32 ? suffix_min_inplace<uint32_t>(t->pos[l], t->npos[l], stream)
