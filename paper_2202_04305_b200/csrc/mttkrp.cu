@@ -17,7 +17,10 @@
 
 namespace {
 
-constexpr int kTThreads = 256;
+#ifndef SP_MTTKRP_THREADS
+#define SP_MTTKRP_THREADS 256
+#endif
+constexpr int kTThreads = SP_MTTKRP_THREADS;
 constexpr int kTPer = 512;   // entries per warp
 
 // One nnz batch = up to 32 consecutive entries held one per lane (coordinate, value).

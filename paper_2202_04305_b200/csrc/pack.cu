@@ -578,22 +578,24 @@ k_count_flags(const uint64_t* __restrict__ keys, int64_t n, LevelPlan p, uint64_
 static_assert(kField * SP_MAX_RANK <= 64 && (1 << kField) > kCtTile, "packed per-tile counters");
 
 // One block (512 threads) per level: tilesum (packed) -> tileprefix[l][tile] (exclusive), counts[l].
-// Across tiles the counts outgrow the packed fields, so each level is scanned on its own.
+// Across tiles the counts outgrow the packed fields, so each level is scanned on its own.  A thread
+// owns a run of consecutive tiles, so the block scans once however many tiles there are.
 __global__ void __launch_bounds__(512)
 k_scan_tiles(const uint64_t* __restrict__ tilesum, int64_t ntiles, int rank, int64_t* __restrict__ tileprefix,
              int64_t* __restrict__ counts) {
     __shared__ uint64_t sums[16];
+    const int64_t per = (ntiles + 511) / 512;
+    const int64_t q0 = (int64_t)threadIdx.x * per, q1 = q0 + per < ntiles ? q0 + per : ntiles;
     for (int l = blockIdx.x; l < rank; l += gridDim.x) {
-        uint64_t run = 0;
-        for (int64_t base = 0; base < ntiles; base += 512) {
-            const int64_t i = base + threadIdx.x;
-            const uint64_t v = i < ntiles ? ((tilesum[i] >> (kField * l)) & kFieldMask) : 0;
-            uint64_t tot;
-            const uint64_t ex = block_excl_scan64(v, sums, &tot);
-            if (i < ntiles) tileprefix[(int64_t)l * ntiles + i] = (int64_t)(run + ex);
-            run += tot;
+        uint64_t local = 0;
+        for (int64_t q = q0; q < q1; ++q) local += (tilesum[q] >> (kField * l)) & kFieldMask;
+        uint64_t tot;
+        uint64_t run = block_excl_scan64(local, sums, &tot);
+        for (int64_t q = q0; q < q1; ++q) {
+            tileprefix[(int64_t)l * ntiles + q] = (int64_t)run;
+            run += (tilesum[q] >> (kField * l)) & kFieldMask;
         }
-        if (threadIdx.x == 0) counts[l] = (int64_t)run;
+        if (threadIdx.x == 0) counts[l] = (int64_t)tot;
     }
 }
 
@@ -630,9 +632,7 @@ struct EmitArgs {
 // the warps total their flags per level, then (the totals exchanged through shared memory) each entry
 // gets its ids from the same ballots and walks its levels on its own.
 // W32: positions and coordinates are stored as 32-bit words (plain stores instead of a width switch).
-// ALLC: every level is compressed, so a node's parent position is the parent's node id and "my parent
-// is new" is the previous level's flag: no linearised positions, no look at the previous key.
-template <int RANK, bool W32, bool ALLC>
+template <int RANK, bool W32>
 __global__ void SP_EMIT_BOUNDS k_emit(EmitArgs a) {
     __shared__ uint32_t wtot[kCtThreads / 32][SP_MAX_RANK];
     const LevelPlan& p = a.plan;
@@ -703,19 +703,22 @@ __global__ void SP_EMIT_BOUNDS k_emit(EmitArgs a) {
         int hb_next = __shfl_down_sync(0xffffffffu, hb[i], 1);
         const int hb_wrap = __shfl_sync(0xffffffffu, hb[i + 1 < kCtIpt ? i + 1 : i], 0);
         if (lane == 31) hb_next = i + 1 < kCtIpt ? hb_wrap : ((e + 1 < a.n && knext == k[i]) ? 0 : 64);
-        int64_t ppos = 0;
-        bool full = false;
-        if (ALLC) {
-            uint32_t parent = 0;
-            bool parent_new = e == 0;
+        // Walk the levels.  `parent` is the position of this entry's node one level up: a node id under a
+        // compressed level, parent * size + coordinate under a dense one; it is a new position exactly
+        // when the level above opened a node for this entry (its flag), or for the very first entry.
+        int64_t parent = 0;
+        bool parent_new = e == 0;
 #pragma unroll
-            for (int l = 0; l < RANK; ++l) {
-                const bool fl = hb[i] > p.shift[l];
+        for (int l = 0; l < RANK; ++l) {
+            const bool fl = hb[i] > p.shift[l];                                           // never set past the end
+            const uint64_t c = (k[i] >> p.shift[l]) & (((uint64_t)1 << p.bits[l]) - 1);   // bits[l] <= 63
+            if (p.lt[l] == SP_DENSE) {                                                    // uniform branch
+                parent = parent * p.sz[l] + (int64_t)c;
+            } else {
                 const uint32_t m = __ballot_sync(0xffffffffu, fl);
                 const uint32_t nid = run[l] + (uint32_t)__popc(m & le_mask) - 1u;
                 run[l] += (uint32_t)__popc(m);
-                if (fl) {                              // never set past the end
-                    const uint64_t c = (k[i] >> p.shift[l]) & (((uint64_t)1 << p.bits[l]) - 1);   // bits[l] <= 63
+                if (fl) {
                     if (W32) static_cast<uint32_t*>(a.crd[l])[nid] = (uint32_t)c;
                     else sp_store_uint(a.crd[l], nid, c, a.crdBits);
                     if (parent_new) {
@@ -724,42 +727,11 @@ __global__ void SP_EMIT_BOUNDS k_emit(EmitArgs a) {
                     }
                 }
                 parent = nid;
-                parent_new = fl;
             }
-            full = parent_new;
-            ppos = parent;
-        } else {
-            const uint64_t kp = prev_key(i);
-            int64_t pprev = 0;
-#pragma unroll
-            for (int l = 0; l < RANK; ++l) {
-                const bool fl = hb[i] > p.shift[l];
-                const uint32_t m = __ballot_sync(0xffffffffu, fl);
-                const int64_t incl = (int64_t)(run[l] + (uint32_t)__popc(m & le_mask));
-                run[l] += (uint32_t)__popc(m);
-                if (e >= a.n) continue;
-                const uint64_t mask = p.bits[l] >= 64 ? ~0ull : ((1ull << p.bits[l]) - 1);
-                const int64_t c = (int64_t)((k[i] >> p.shift[l]) & mask);
-                if (l == RANK - 1) full = fl;
-                if (p.lt[l] == SP_DENSE) {
-                    const int64_t cp = (int64_t)((kp >> p.shift[l]) & mask);
-                    ppos = ppos * p.sz[l] + c;
-                    pprev = pprev * p.sz[l] + cp;
-                } else {
-                    const int64_t nid = incl - 1;
-                    if (fl) {
-                        if (W32) static_cast<uint32_t*>(a.crd[l])[nid] = (uint32_t)c;
-                        else sp_store_uint(a.crd[l], nid, (uint64_t)c, a.crdBits);
-                        if (e == 0 || pprev != ppos) {
-                            if (W32) static_cast<uint32_t*>(a.pos[l])[ppos] = (uint32_t)nid;
-                            else sp_store_uint(a.pos[l], ppos, (uint64_t)nid, a.posBits);
-                        }
-                    }
-                    pprev = nid - (fl ? 1 : 0);
-                    ppos = nid;
-                }
-            }
+            parent_new = fl;
         }
+        const bool full = parent_new;
+        const int64_t ppos = parent;
         if (e >= a.n) continue;
         if (full) {
             double s = vin[i];
@@ -984,12 +956,11 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         // every buffer of the pack in one allocation
         ws.reserve(2 * sp_workspace::bytes_for<uint64_t>((size_t)n) +
                    (fused ? sp_workspace::bytes_for<uint32_t>((size_t)n) : npasses > 0 ? 2 * sp_workspace::bytes_for<uint64_t>((size_t)n) : 0) +
-                   sp_workspace::bytes_for<int>(1) + sp_workspace::bytes_for<uint32_t>((size_t)stiles << kMaxDigitBits) +
+                   sp_workspace::bytes_for<uint32_t>((size_t)stiles << kMaxDigitBits) +
                    sp_workspace::bytes_for<uint32_t>((size_t)1 << kMaxDigitBits) + sp_workspace::bytes_for<uint32_t>(nscan) +
                    sp_workspace::bytes_for<uint64_t>((size_t)ct_tiles) + sp_workspace::bytes_for<int64_t>((size_t)ct_tiles * SP_MAX_RANK) +
-                   sp_workspace::bytes_for<int64_t>(SP_MAX_RANK));
+                   sp_workspace::bytes_for<int64_t>(SP_MAX_RANK + 1));
         uint64_t* kbuf[2] = {ws.get<uint64_t>((size_t)n), ws.get<uint64_t>((size_t)n)};
-        d_err = ws.get<int>(1);
         uint64_t* pbuf[2] = {nullptr, nullptr};
         uint32_t* isorted = nullptr;
         if (fused) isorted = ws.get<uint32_t>((size_t)n);
@@ -999,9 +970,10 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         uint32_t* chunk_tot = ws.get<uint32_t>(nscan);
         uint64_t* tilesum = ws.get<uint64_t>((size_t)ct_tiles);
         tileprefix = ws.get<int64_t>((size_t)ct_tiles * SP_MAX_RANK);
-        int64_t* d_counts = ws.get<int64_t>(SP_MAX_RANK);
+        int64_t* d_counts = ws.get<int64_t>(SP_MAX_RANK + 1);      // node counts per level, then the error word
         if (ws.failed) return SP_ERR_ALLOC;
-        SP_CUDA(cudaMemsetAsync(d_err, 0, sizeof(int), stream));
+        d_err = reinterpret_cast<int*>(d_counts + SP_MAX_RANK);
+        SP_CUDA(cudaMemsetAsync(d_err, 0, sizeof(int64_t), stream));
 
         LevelCoords lc;
         for (int l = 0; l < SP_MAX_RANK; ++l) lc.p[l] = coo_coords[l < rank ? plan.src[l] : 0];
@@ -1059,10 +1031,11 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         SP_LAUNCH_CHECK();
         timer.mark(kPhCount);
         sp_count_launches(3);
-        int h_err = 0;
-        SP_CUDA(cudaMemcpyAsync(counts, d_counts, sizeof counts, cudaMemcpyDeviceToHost, stream));
-        SP_CUDA(cudaMemcpyAsync(&h_err, d_err, sizeof h_err, cudaMemcpyDeviceToHost, stream));
+        int64_t h_back[SP_MAX_RANK + 1] = {};          // one read-back: the counts and the error word
+        SP_CUDA(cudaMemcpyAsync(h_back, d_counts, sizeof h_back, cudaMemcpyDeviceToHost, stream));
         SP_CUDA(cudaStreamSynchronize(stream));
+        for (int l = 0; l < SP_MAX_RANK; ++l) counts[l] = h_back[l];
+        const int h_err = (int)(h_back[SP_MAX_RANK] & 0xffffffff);
         if (h_err & kErrRange) return SP_ERR_OUT_OF_RANGE;
         if ((flags & SP_DUP_ERROR) && counts[rank - 1] != n) return SP_ERR_DUPLICATE;
     }
@@ -1149,17 +1122,10 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
             t->parts[(uint64_t)SP_PART_SEGIDS << 56] = sg;
         }
         const bool w32 = posBits == 32 && crdBits == 32;
-        bool allc = true;
-        for (int l = 0; l < rank; ++l) allc = allc && plan.lt[l] == SP_COMPRESSED;
 #define SP_EMIT(R)                                                                              \
     case R:                                                                                     \
-        if (allc) {                                                                             \
-            if (w32) k_emit<R, true, true><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);   \
-            else k_emit<R, false, true><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);      \
-        } else {                                                                                \
-            if (w32) k_emit<R, true, false><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);  \
-            else k_emit<R, false, false><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);     \
-        }                                                                                       \
+        if (w32) k_emit<R, true><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);             \
+        else k_emit<R, false><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(a);                \
         break;
         switch (rank) { SP_EMIT(1) SP_EMIT(2) SP_EMIT(3) SP_EMIT(4) SP_EMIT(5) }
 #undef SP_EMIT
