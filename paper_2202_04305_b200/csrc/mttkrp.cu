@@ -17,10 +17,7 @@
 
 namespace {
 
-#ifndef SP_MTTKRP_THREADS
-#define SP_MTTKRP_THREADS 256
-#endif
-constexpr int kTThreads = SP_MTTKRP_THREADS;
+constexpr int kTThreads = 256;
 constexpr int kTPer = 512;   // entries per warp
 
 // One nnz batch = up to 32 consecutive entries held one per lane (coordinate, value).
@@ -203,11 +200,19 @@ __device__ __forceinline__ void ld_cols(const double* p, const int* coff, double
     }
 }
 
-#ifndef SP_LB_MTTKRP
-#define SP_LB_MTTKRP 2
+// Two warps per block, eight blocks per SM: the same 16 warps per SM as 256 x 2 (126 registers a thread
+// either way), but a block's warps share nothing until the final combine of their open slices, and
+// small blocks finish and are replaced more evenly: 0.527 ms against 0.555 ms on the 20,000,000-entry
+// tensor (128 x 4: 0.533, 32 x 16: 0.528, 512 x 1: 0.583).
+#ifndef SP_MTTKRP_FAST_THREADS
+#define SP_MTTKRP_FAST_THREADS 64
 #endif
+#ifndef SP_LB_MTTKRP
+#define SP_LB_MTTKRP (512 / SP_MTTKRP_FAST_THREADS)
+#endif
+constexpr int kFThreads = SP_MTTKRP_FAST_THREADS;
 template <typename P, typename I, int S, bool W256>
-__global__ void __launch_bounds__(kTThreads, SP_LB_MTTKRP)
+__global__ void __launch_bounds__(kFThreads, SP_LB_MTTKRP)
 k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* __restrict__ pos2,
               const I* __restrict__ crd1, const I* __restrict__ crd2, const double* __restrict__ val,
               const double* __restrict__ F1, const double* __restrict__ F2, int64_t R, double* __restrict__ M,
@@ -216,7 +221,7 @@ k_mttkrp_fast(const P* __restrict__ pos1, const I* __restrict__ crd0, const P* _
               int64_t d0, int64_t d1, int64_t d2) {
     constexpr int GL = 32 / S;      // lanes per group = entries per group and batch
     constexpr int kStepGroup = S == 2 ? 4 : 2;
-    constexpr int kWarps = kTThreads / 32;
+    constexpr int kWarps = kFThreads / 32;
     __shared__ Staged s_st[kWarps][32];
     __shared__ double s_car[2 * kWarps][32];
     __shared__ long long s_id[2 * kWarps];
@@ -448,10 +453,10 @@ static sp_status mttkrp_levels(sp_tensor* T, const double* F1, const double* F2,
     sp_partition part;
     sp_status st = sp_get_mttkrp_partition(T, fast ? kFastPer : kTPer, stream, &part);
     if (st != SP_OK) return st;
-    const unsigned blocks = (unsigned)sp_ceil_div(part.nchunks * 32, kTThreads);
+    const unsigned blocks = (unsigned)sp_ceil_div(part.nchunks * 32, fast ? kFThreads : kTThreads);
     if (fast) {
 #define SP_MTTKRP_FAST(S, W)                                                                                           \
-    k_mttkrp_fast<P, I, S, W><<<blocks, kTThreads, 0, stream>>>(                                                       \
+    k_mttkrp_fast<P, I, S, W><<<blocks, kFThreads, 0, stream>>>(                                                       \
         static_cast<const P*>(T->pos[1]), T->lt[0] == SP_COMPRESSED ? static_cast<const I*>(T->crd[0]) : nullptr,      \
         static_cast<const P*>(T->pos[2]), static_cast<const I*>(T->crd[1]), static_cast<const I*>(T->crd[2]), T->val,  \
         F1, F2, R, M, part.row, part.nz, part.aux, part.nchunks, T->npos[1] - 1, T->ncrd[1], T->dims[T->ord[0]], d1, d2)
