@@ -190,8 +190,11 @@ __global__ void k_spmv_fixup(const double* __restrict__ carry_val, const int64_t
 // Rows without entries (CSR) are written as zeros here; when level 0 is compressed the group of
 // stored row q also writes the zeros of the rows that storage elides between stored rows q - 1 and q
 // (the last group those after its row too), so y needs no clearing pass.
+#ifndef SP_SPMV_ROWS_THREADS
+#define SP_SPMV_ROWS_THREADS 64
+#endif
 template <typename P, typename I, int G>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(SP_SPMV_ROWS_THREADS)
 k_spmv_rows(const P* __restrict__ pos, const I* __restrict__ crd, const double* __restrict__ val,
             const I* __restrict__ outer, const double* __restrict__ x, double* __restrict__ y, int64_t nseg,
             int64_t m, int64_t n, int64_t nnz) {
@@ -369,7 +372,7 @@ k_spmm_gather(const P* __restrict__ pos, const I* __restrict__ crd, const double
 // compressed the group of stored row q also writes the zeros of the rows that storage elides between
 // stored rows q - 1 and q (the last group those after its row too), so that C needs no clearing pass.
 #ifndef SP_SPMM_ROWS_THREADS
-#define SP_SPMM_ROWS_THREADS 256
+#define SP_SPMM_ROWS_THREADS 64
 #endif
 #ifdef SP_LB_ROWS
 #define SP_ROWS_BOUNDS __launch_bounds__(SP_SPMM_ROWS_THREADS, SP_LB_ROWS)
@@ -556,15 +559,15 @@ extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* str
             // rows of mean 16 and up to 435 entries, 16 lanes 0.023 ms, 4 lanes 0.031.
             const int64_t want = std::max<int64_t>(mean / 6, max_seg / 32);
             const int G = want <= 4 ? 4 : (want <= 8 ? 8 : (want <= 16 ? 16 : 32));
-            const unsigned blocks = (unsigned)sp_ceil_div(nseg * G, 256);
+            const unsigned blocks = (unsigned)sp_ceil_div(nseg * G, SP_SPMV_ROWS_THREADS);
             SP_DISPATCH_WIDTHS(A, {
                 const P* pos = static_cast<const P*>(A->pos[1]);
                 const I* crd = static_cast<const I*>(A->crd[1]);
                 const I* outer = dbl ? static_cast<const I*>(A->crd[0]) : nullptr;
-                if (G == 4) k_spmv_rows<P, I, 4><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg, m, A->dims[1], A->ncrd[1]);
-                else if (G == 8) k_spmv_rows<P, I, 8><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg, m, A->dims[1], A->ncrd[1]);
-                else if (G == 16) k_spmv_rows<P, I, 16><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg, m, A->dims[1], A->ncrd[1]);
-                else k_spmv_rows<P, I, 32><<<blocks, 256, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg, m, A->dims[1], A->ncrd[1]);
+                if (G == 4) k_spmv_rows<P, I, 4><<<blocks, SP_SPMV_ROWS_THREADS, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg, m, A->dims[1], A->ncrd[1]);
+                else if (G == 8) k_spmv_rows<P, I, 8><<<blocks, SP_SPMV_ROWS_THREADS, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg, m, A->dims[1], A->ncrd[1]);
+                else if (G == 16) k_spmv_rows<P, I, 16><<<blocks, SP_SPMV_ROWS_THREADS, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg, m, A->dims[1], A->ncrd[1]);
+                else k_spmv_rows<P, I, 32><<<blocks, SP_SPMV_ROWS_THREADS, 0, stream>>>(pos, crd, A->val, outer, x, y, nseg, m, A->dims[1], A->ncrd[1]);
             });
             SP_LAUNCH_CHECK();
             sp_count_launches(1);
