@@ -784,7 +784,11 @@ def main():
                     "achieved": round(ach, 1), "peak": peak, "unit": "GB/s", "frac": round(ach / peak, 4),
                     "peak_kind": f"of {peak_kind}",
                     "traffic": NCU_TRAFFIC.get("k_sort_downsweep") if n5 == 20_000_000 else None,
-                    "algorithmic_bytes_per_launch": per_entry * n5, "launch_ms": round(sc_ms, 4)}
+                    "algorithmic_bytes_per_launch": per_entry * n5, "launch_ms": round(sc_ms, 4),
+                    # the same launch time against the 24 B per entry of a pass that carries a 4-byte entry
+                    # index instead of the 8-byte value (that design needs a value gather at the end of the
+                    # pack, which cost more than the six passes' extra 8 bytes: 1.68 ms per pack against 1.43)
+                    "frac_if_counted_at_24B_per_entry": round(24 * n5 / (sc_ms * 1e-3) / 1e9 / peak, 4)}
     else:
         kk = kernels[dominant]
         roofline = {"kernel": dominant, "bound": "hbm", "achieved": kk["eff_gbs"], "peak": peak, "unit": "GB/s",
