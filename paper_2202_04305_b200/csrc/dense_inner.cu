@@ -20,7 +20,7 @@ constexpr int kDUnroll = 8;
 template <typename I, int TPR>
 __global__ void __launch_bounds__(kDThreads)
 k_spmv_dense_rows(const double* __restrict__ val, const I* __restrict__ outer, int64_t nslices, int64_t inner,
-                  const double* __restrict__ x, double* __restrict__ y) {
+                  const double* __restrict__ x, double* __restrict__ y, int64_t douter) {
     __shared__ double s_part[kDThreads / 32];
     constexpr int kGroups = kDThreads / TPR;
     const int g = threadIdx.x / TPR, tl = threadIdx.x % TPR;
@@ -56,7 +56,7 @@ k_spmv_dense_rows(const double* __restrict__ val, const I* __restrict__ outer, i
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
         if (TPR == 32) {
-            if (tl == 0) y[outer ? (int64_t)outer[q] : q] = s;
+            if (tl == 0) y[SP_IDX(outer ? (int64_t)outer[q] : q, douter)] = s;
         } else {                                  // TPR == kDThreads: the whole block works on slice q
             if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = s;
             __syncthreads();
@@ -64,7 +64,7 @@ k_spmv_dense_rows(const double* __restrict__ val, const I* __restrict__ outer, i
                 double tot = s_part[0];
 #pragma unroll
                 for (int i = 1; i < kDThreads / 32; ++i) tot += s_part[i];
-                y[outer ? (int64_t)outer[q] : q] = tot;
+                y[SP_IDX(outer ? (int64_t)outer[q] : q, douter)] = tot;
             }
             __syncthreads();
         }
@@ -76,13 +76,13 @@ constexpr int kDChunk = 32;
 template <typename I>
 __global__ void __launch_bounds__(kDThreads)
 k_spmv_dense_cols(const double* __restrict__ val, const I* __restrict__ outer, int64_t nslices, int64_t inner,
-                  const double* __restrict__ x, double* __restrict__ y) {
+                  const double* __restrict__ x, double* __restrict__ y, int64_t douter) {
     const int64_t i = (int64_t)blockIdx.x * kDThreads + threadIdx.x;
     if (i >= inner) return;
     const int64_t q0 = (int64_t)blockIdx.y * kDChunk;
     const int64_t q1 = q0 + kDChunk < nslices ? q0 + kDChunk : nslices;
     double s = 0.0;
-    for (int64_t q = q0; q < q1; ++q) s = fma(__ldcs(val + q * inner + i), __ldg(x + (outer ? (int64_t)outer[q] : q)), s);
+    for (int64_t q = q0; q < q1; ++q) s = fma(__ldcs(val + q * inner + i), __ldg(x + SP_IDX(outer ? (int64_t)outer[q] : q, douter)), s);
     atomicAdd(y + i, s);
 }
 
@@ -111,7 +111,7 @@ template <typename I, bool ROWMAJOR>
 __global__ void __launch_bounds__(kDThreads, 2)
 k_spmm_dense_inner(const double* __restrict__ val, const I* __restrict__ outer, int64_t nslices, int64_t inner,
                    const double* __restrict__ B, int64_t N, int64_t ldb, double* __restrict__ C, int64_t ldc,
-                   int64_t kchunk, int vec_a) {
+                   int64_t kchunk, int vec_a, int64_t douter) {
     __shared__ __align__(16) double s_a[2][kKT][kAStride];
     __shared__ __align__(16) double s_b[2][kKT][kBStride];
     const int t = threadIdx.x, lane = t & 31, w = t >> 5;
@@ -156,7 +156,7 @@ k_spmm_dense_inner(const double* __restrict__ val, const I* __restrict__ outer, 
         }
         const int64_t k = k0 + bk, c = c0 + bc;
         b_reg = 0.0;
-        if (k < kend && c < N) b_reg = __ldg(B + (ROWMAJOR ? k : (outer ? (int64_t)outer[k] : k)) * ldb + c);
+        if (k < kend && c < N) b_reg = __ldg(B + (ROWMAJOR ? k : SP_IDX(outer ? (int64_t)outer[k] : k, douter)) * ldb + c);
     };
     auto store_tile = [&](int buf) {
         if (quad) {
@@ -209,7 +209,7 @@ k_spmm_dense_inner(const double* __restrict__ val, const I* __restrict__ outer, 
     for (int i = 0; i < 4; ++i) {
         const int64_t row = r0 + w * 32 + i * 8 + fr;
         if (row >= nrows) continue;
-        double* dst = C + (ROWMAJOR ? (outer ? (int64_t)outer[row] : row) : row) * ldc;
+        double* dst = C + (ROWMAJOR ? SP_IDX(outer ? (int64_t)outer[row] : row, douter) : row) * ldc;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
 #pragma unroll
@@ -292,7 +292,7 @@ template <typename I>
 __global__ void __launch_bounds__(kTThreads, SP_TMA_BLOCKS)
 k_spmm_dense_inner_tma(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                        const I* __restrict__ outer, int64_t nrows, int64_t nk, int64_t N, double* __restrict__ C,
-                       int64_t ldc, int64_t kchunk, int* __restrict__ gave_up) {
+                       int64_t ldc, int64_t kchunk, int* __restrict__ gave_up, int64_t douter) {
     extern __shared__ __align__(128) unsigned char s_raw[];
     double* s_stage = reinterpret_cast<double*>((reinterpret_cast<uintptr_t>(s_raw) + 127) & ~(uintptr_t)127);
     uint64_t* s_full = reinterpret_cast<uint64_t*>(s_stage + (size_t)kTStages * kStageDoubles);
@@ -371,7 +371,7 @@ k_spmm_dense_inner_tma(const __grid_constant__ CUtensorMap map_a, const __grid_c
     for (int i = 0; i < 4; ++i) {
         const int64_t row = (int64_t)r0 + w * 32 + i * 8 + fr;
         if (row >= nrows) continue;
-        double* dst = C + (outer ? (int64_t)outer[row] : row) * ldc;
+        double* dst = C + SP_IDX(outer ? (int64_t)outer[row] : row, douter) * ldc;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
 #pragma unroll
@@ -480,12 +480,13 @@ sp_status spmm_dense_inner_tma(const sp_tensor* A, const void* outer, int64_t ns
     }
     if (wi == 0)
         k_spmm_dense_inner_tma<uint32_t><<<grid, kTThreads, kTmaSmem, stream>>>(map_a, map_b, static_cast<const uint32_t*>(outer), nslices,
-                                                                                inner, N, C, ldc, kchunk, h.gave_up_dev);
+                                                                                inner, N, C, ldc, kchunk, h.gave_up_dev, A->dims[A->ord[0]]);
     else
         k_spmm_dense_inner_tma<uint64_t><<<grid, kTThreads, kTmaSmem, stream>>>(map_a, map_b, static_cast<const uint64_t*>(outer), nslices,
-                                                                                inner, N, C, ldc, kchunk, h.gave_up_dev);
+                                                                                inner, N, C, ldc, kchunk, h.gave_up_dev, A->dims[A->ord[0]]);
     SP_LAUNCH_CHECK();
     sp_count_launches(1);
+    SP_BOUNDS_RETURN(stream);
     return SP_OK;
 }
 
@@ -506,23 +507,24 @@ sp_status sp_spmv_dense_inner(const sp_tensor* A, const double* x, double* y, cu
         if (rowmajor) {                                                                                              \
             if (inner >= 1024) {                                                                                     \
                 const unsigned blocks = (unsigned)(nslices < 148 * 16 ? nslices : 148 * 16);                         \
-                k_spmv_dense_rows<I, kDThreads><<<blocks, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, x, y); \
+                k_spmv_dense_rows<I, kDThreads><<<blocks, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, x, y, A->dims[A->ord[0]]); \
             } else {                                                                                                 \
                 const int64_t need = sp_ceil_div(nslices, kDThreads / 32);                                           \
                 const unsigned blocks = (unsigned)(need < 148 * 16 ? need : 148 * 16);                               \
-                k_spmv_dense_rows<I, 32><<<blocks, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, x, y);     \
+                k_spmv_dense_rows<I, 32><<<blocks, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, x, y, A->dims[A->ord[0]]);     \
             }                                                                                                        \
         } else {                                                                                                     \
             const int64_t chunks = sp_ceil_div(nslices, kDChunk);                                                    \
             if (chunks > 65535) return SP_ERR_UNSUPPORTED;                                                           \
             dim3 grid((unsigned)sp_ceil_div(inner, kDThreads), (unsigned)chunks);                                    \
-            k_spmv_dense_cols<I><<<grid, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, x, y);               \
+            k_spmv_dense_cols<I><<<grid, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, x, y, A->dims[A->ord[0]]);               \
         }                                                                                                            \
     } while (0)
     if (A->crdBits == 32) SP_DENSE_LAUNCH(uint32_t); else SP_DENSE_LAUNCH(uint64_t);
 #undef SP_DENSE_LAUNCH
     SP_LAUNCH_CHECK();
     sp_count_launches(1);
+    SP_BOUNDS_RETURN(stream);
     return SP_OK;
 }
 
@@ -571,12 +573,13 @@ sp_status sp_spmm_dense_inner(const sp_tensor* A, const double* B, int64_t N, in
 #define SP_DENSE_MM(I)                                                                                                  \
     do {                                                                                                                \
         const I* outer = outer_c ? static_cast<const I*>(A->crd[0]) : nullptr;                                          \
-        if (rowmajor) k_spmm_dense_inner<I, true><<<grid, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, B, N, ldb, C, ldc, kchunk, vec_a); \
-        else k_spmm_dense_inner<I, false><<<grid, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, B, N, ldb, C, ldc, kchunk, vec_a);       \
+        if (rowmajor) k_spmm_dense_inner<I, true><<<grid, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, B, N, ldb, C, ldc, kchunk, vec_a, A->dims[A->ord[0]]); \
+        else k_spmm_dense_inner<I, false><<<grid, kDThreads, 0, stream>>>(A->val, outer, nslices, inner, B, N, ldb, C, ldc, kchunk, vec_a, A->dims[A->ord[0]]);       \
     } while (0)
     if (A->crdBits == 32) SP_DENSE_MM(uint32_t); else SP_DENSE_MM(uint64_t);
 #undef SP_DENSE_MM
     SP_LAUNCH_CHECK();
     sp_count_launches(1);
+    SP_BOUNDS_RETURN(stream);
     return SP_OK;
 }

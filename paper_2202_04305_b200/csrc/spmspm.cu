@@ -49,7 +49,7 @@ k_spmspm(const P* __restrict__ apos, const I* __restrict__ acrd, const double* _
          const P* __restrict__ bpos, const I* __restrict__ bcrd, const double* __restrict__ bval, int64_t m,
          int64_t n, double* __restrict__ ws_all, uint32_t* __restrict__ bm_all, int64_t* __restrict__ rowlen,
          const void* __restrict__ cpos, int cposBits, void* __restrict__ ccrd, int ccrdBits,
-         double* __restrict__ cval) {
+         double* __restrict__ cval, int64_t kdim) {
     __shared__ uint32_t sums[kPThreads / 32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int64_t words = (n + 31) >> 5;
@@ -72,11 +72,11 @@ k_spmspm(const P* __restrict__ apos, const I* __restrict__ acrd, const double* _
         // expand: every product of row i lands in the workspace
         const int64_t a0 = (int64_t)apos[i], a1 = (int64_t)apos[i + 1];
         for (int64_t p = a0 + w; p < a1; p += kPThreads / 32) {
-            const int64_t k = (int64_t)acrd[p];
+            const int64_t k = SP_IDX((int64_t)acrd[p], kdim);
             const double a = aval[p];
             const int64_t b0 = (int64_t)bpos[k], b1 = (int64_t)bpos[k + 1];
             for (int64_t q = b0 + lane; q < b1; q += 32) {
-                const int64_t j = (int64_t)bcrd[q];
+                const int64_t j = SP_IDX((int64_t)bcrd[q], n);
                 atomicOr(bm + (j >> 5), 1u << (j & 31));
                 if (NUMERIC) atomicAdd(ws + j, a * bval[q]);
             }
@@ -229,7 +229,8 @@ extern "C" sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBi
 
 #define SP_SPMSPM_ARGS                                                                                            \
     static_cast<const P*>(A->pos[1]), static_cast<const I*>(A->crd[1]), A->val, static_cast<const P*>(B->pos[1]), \
-        static_cast<const I*>(B->crd[1]), B->val, m, n, wsrow, bm, rowlen, C->pos[1], posBits, C->crd[1], crdBits, C->val
+        static_cast<const I*>(B->crd[1]), B->val, m, n, wsrow, bm, rowlen, C->pos[1], posBits, C->crd[1], crdBits, C->val, \
+        B->dims[0]
 #define SP_SPMSPM_LAUNCH(NUM)                                                                                     \
     SP_DISPATCH_WIDTHS(A, {                                                                                       \
         if (in_smem) {                                                                                            \
@@ -263,6 +264,9 @@ extern "C" sp_status sp_spmspm(const sp_tensor* A, const sp_tensor* B, int posBi
     }
 #undef SP_SPMSPM_LAUNCH
 #undef SP_SPMSPM_ARGS
+#ifdef SP_DEBUG_BOUNDS
+    { const sp_status b = sp_bounds_result(stream); if (b != SP_OK) return fail(b); }
+#endif
     *out = C;
     return SP_OK;
 }

@@ -60,6 +60,24 @@ for lt in [(1, 1, 1), (0, 1, 1)]:
     T = sp.sp_pack(t.dims, tc, tv, lt)
     assert_close(sp.sp_mttkrp(T, dev(Bf), dev(Cf)).cpu().numpy(), Mref, Mb, f"mttkrp {lt}")
 
+# dense inner level (both feeds of the SpMM, SpMV, SDDMM) and the all-sparse product
+small = I.uniform_matrix(300, 260, 9000, seed=5)
+sc, sv = to_dev(small)
+Bs, xs = I.dense_operand(5, 31, 260, 12), I.uniform_pm1(5, 32, 260)
+Cs, Csb = O.spmm(300, small.coords[0], small.coords[1], small.vals, Bs)
+ys, ysb = O.spmv(300, small.coords[0], small.coords[1], small.vals, xs)
+for lt, od in [((1, 0), (0, 1)), ((0, 0), (0, 1)), ((1, 0), (1, 0))]:
+    A = sp.sp_pack(small.dims, sc, sv, lt, od)
+    assert_close(sp.sp_spmm(A, dev(Bs)).cpu().numpy(), Cs, Csb, f"dense inner {lt} {od}")
+    assert_close(sp.sp_spmm(A, dev(Bs[:, :7].copy())).cpu().numpy(), Cs[:, :7], Csb[:, :7], "dense inner, odd width")
+    assert_close(sp.sp_spmv(A, dev(xs)).cpu().numpy(), ys, ysb, f"dense inner spmv {lt} {od}")
+P, Q = I.uniform_matrix(120, 90, 900, seed=6), I.uniform_matrix(90, 150, 1100, seed=7)
+hP, hQ = sp.sp_pack(P.dims, *to_dev(P), (0, 1)), sp.sp_pack(Q.dims, *to_dev(Q), (0, 1))
+hC = sp.sp_spmspm(hP, hQ)
+pos, crdC, valC, bdC = O.spmspm(120, 90, 150, P.coords[0], P.coords[1], P.vals, Q.coords[0], Q.coords[1], Q.vals)
+assert np.array_equal(hC.coordinates(1).cpu().numpy().astype(np.int64), crdC)
+assert_close(hC.values().cpu().numpy(), valC, bdC, "spmspm")
+
 # 2. a coordinate out of range: status 3, no fault; operands hold twice the declared rows
 n = 700
 A = sp.sp_pack(coo.dims, coords, vals, (0, 1))
@@ -78,6 +96,22 @@ for call in (lambda: sp.sp_spmv(A, x2[:n]), lambda: sp.sp_spmm(A, B2[:n])):
 crd[7] = keep
 assert_close(sp.sp_spmv(A, x2[:n]).cpu().numpy(), yref, yb, "after repair")
 assert_close(sp.sp_spmm(A, B2[:n]).cpu().numpy(), Cref, Cb, "after repair")
+
+Ad = sp.sp_pack(small.dims, sc, sv, (1, 0), (0, 1))          # CDR: the stored row numbers address the output
+c0 = Ad.coordinates(0)
+keep = int(c0[3])
+c0[3] = 300 + 2
+Cbig = torch.zeros(2 * 300, 12, dtype=torch.float64, device="cuda")
+ybig = torch.zeros(2 * 300, dtype=torch.float64, device="cuda")
+for call in (lambda: sp.sp_spmm(Ad, dev(Bs), Cbig[:300]), lambda: sp.sp_spmv(Ad, dev(xs), ybig[:300])):
+    try:
+        call()
+    except sp.SpError as e:
+        assert e.code == 3, e.code
+    else:
+        raise AssertionError("the bad row number went unnoticed")
+c0[3] = keep
+assert_close(sp.sp_spmm(Ad, dev(Bs), Cbig[:300]).cpu().numpy(), Cs, Csb, "dense inner after repair")
 
 T = sp.sp_pack(t.dims, tc, tv, (1, 1, 1))
 C2 = torch.zeros(2 * 96, 8, dtype=torch.float64, device="cuda"); C2[:96] = dev(Cf)
