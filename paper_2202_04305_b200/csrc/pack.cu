@@ -648,6 +648,18 @@ __global__ void SP_EMIT_BOUNDS k_emit(EmitArgs a) {
     }
     if (blockIdx.x == 0 && threadIdx.x < RANK && p.lt[threadIdx.x] == SP_COMPRESSED)   // pos[l] ends with the node count
         sp_store_uint(a.pos[threadIdx.x], a.last_pos[threadIdx.x], (uint64_t)a.last_val[threadIdx.x], a.posBits);
+    // this thread's values, requested before anything is computed
+    double vin[kCtIpt];
+    if (a.vals_sorted) {
+#pragma unroll
+        for (int i = 0; i < kCtIpt; ++i) { const int64_t e = chunk + i * 32 + lane; vin[i] = e < a.n ? a.vals_sorted[e] : 0.0; }
+    } else {
+        uint32_t id[kCtIpt];
+#pragma unroll
+        for (int i = 0; i < kCtIpt; ++i) { const int64_t e = chunk + i * 32 + lane; id[i] = e < a.n ? a.idx[e] : 0u; }
+#pragma unroll
+        for (int i = 0; i < kCtIpt; ++i) vin[i] = a.vals_in[id[i]];
+    }
     const uint64_t kbefore = (chunk > 0 && chunk <= a.n) ? a.keys[chunk - 1] : 0;   // uniform per warp
     // key of the entry before entry (i, lane)
     auto prev_key = [&](int i) -> uint64_t {
@@ -674,18 +686,6 @@ __global__ void SP_EMIT_BOUNDS k_emit(EmitArgs a) {
         for (int l = 0; l < RANK; ++l) wtot[w][l] = tot[l];
     }
 
-    // this thread's values, requested before the barrier
-    double vin[kCtIpt];
-    if (a.vals_sorted) {
-#pragma unroll
-        for (int i = 0; i < kCtIpt; ++i) { const int64_t e = chunk + i * 32 + lane; vin[i] = e < a.n ? a.vals_sorted[e] : 0.0; }
-    } else {
-        uint32_t id[kCtIpt];
-#pragma unroll
-        for (int i = 0; i < kCtIpt; ++i) { const int64_t e = chunk + i * 32 + lane; id[i] = e < a.n ? a.idx[e] : 0u; }
-#pragma unroll
-        for (int i = 0; i < kCtIpt; ++i) vin[i] = a.vals_in[id[i]];
-    }
     __syncthreads();
 
     uint32_t run[RANK];                           // flagged entries at level l before this warp's round (< nnz < 2^32)
