@@ -97,3 +97,33 @@ def test_random_tensors(oracle, block):
         Mr, Mb = oracle.mttkrp(dims[mode], c.coords[mode], c.coords[rs[0]], c.coords[rs[1]], c.vals, F[rs[0]], F[rs[1]])
         Mg = sp().sp_mttkrp_mode(T, mode, [dev(f) for f in F]).cpu().numpy()
         assert_close(Mg, Mr, Mb, "mttkrp " + what)
+
+
+def test_random_dense_inner_products(oracle):
+    """Row bands and full matrices stored with a dense inner level, random sizes, widths N, paddings of B
+    and starts of B on or off a 16-byte boundary: the copy-engine feed and the register-staged feed of
+    sp_spmm, chosen by those alignments, against the oracle; what lies beside B and C stays out of it."""
+    import torch
+    rng = np.random.default_rng(3000)
+    for _ in range(24):
+        seed = int(rng.integers(1, 1 << 30))
+        m, n = int(rng.integers(1, 1500)), int(rng.integers(1, 1500))
+        rows = int(rng.integers(1, min(m, 300) + 1))
+        N = int(rng.choice([1, 2, 6, 7, 8, 16, 30, 32, 33, 40, 64, 70]))
+        ldb, shift = N + int(rng.integers(0, 4)), int(rng.integers(0, 2))
+        cdr = rng.random() < 0.7
+        cbits = 32 if rng.random() < 0.7 else 64
+        rsel = np.sort(rng.choice(m, rows, replace=False)) if cdr else np.arange(m)
+        e = np.arange(rsel.size * n, dtype=np.int64)
+        coo = I.Coo((m, n), [rsel[e // n], e % n], I.uniform_pm1(seed, 1, e.size))
+        B = I.dense_operand(seed, 3, n, N)
+        ref, bd = oracle.spmm(m, coo.coords[0], coo.coords[1], coo.vals, B)
+        coords, vals = to_dev(coo, cbits)
+        A = sp().sp_pack(coo.dims, coords, vals, (1 if cdr else 0, 0), (0, 1), 32, cbits)
+        flat = torch.full((n * ldb + 2,), 1e300, dtype=torch.float64, device="cuda")
+        Bdev = flat[shift:shift + n * ldb].view(n, ldb)[:, :N]
+        Bdev.copy_(dev(B))
+        Cbig = torch.full((m, N + 2), 7.0, dtype=torch.float64, device="cuda")
+        sp().sp_spmm(A, Bdev, Cbig[:, :N])
+        assert_close(Cbig[:, :N].cpu().numpy(), ref, bd, f"dense inner {(m, n, rows, N, ldb, shift, cdr, cbits)}")
+        assert torch.all(Cbig[:, N:] == 7.0)
