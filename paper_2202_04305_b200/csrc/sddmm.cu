@@ -94,22 +94,50 @@ k_sddmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __re
                 off = 0;
             }
             const int cnt = (int)min(rend - p, (int64_t)(32 - off));
-            for (int t = 0; t < cnt; ++t) {
-                const int64_t j = SP_IDX(__shfl_sync(0xffffffffu, c_l, off + t), nb);
-                const double* brow = Bt + j * ldt;
-                double part = 0.0;
-                if (NCH > 0) {
+#ifndef SP_SDDMM_BATCH
+#define SP_SDDMM_BATCH 2
+#endif
+            if (NCH > 0) {
+                // kB entries at a time: all their operand loads are requested before the first of the
+                // (dependent) warp reductions starts; a batch's tail repeats its last entry
+                constexpr int kB = SP_SDDMM_BATCH;
+                for (int t = 0; t < cnt; t += kB) {
+                    double b[kB][NA][V];
 #pragma unroll
-                    for (int ch = 0; ch < NA; ++ch) {
-                        const int64_t kk = (int64_t)ch * 32 * V + lane * V;
-                        if (kk < K) {
-                            double b[V];
-                            ld2<V>(brow + kk, b);
+                    for (int u = 0; u < kB; ++u) {
+                        const int tt = t + u < cnt ? t + u : cnt - 1;
+                        const int64_t j = SP_IDX(__shfl_sync(0xffffffffu, c_l, off + tt), nb);
+                        const double* brow = Bt + j * ldt;
 #pragma unroll
-                            for (int q = 0; q < V; ++q) part = fma(a[ch][q], b[q], part);
+                        for (int ch = 0; ch < NA; ++ch) {
+                            const int64_t kk = (int64_t)ch * 32 * V + lane * V;
+#pragma unroll
+                            for (int q = 0; q < V; ++q) b[u][ch][q] = 0.0;
+                            if (kk < K) ld2<V>(brow + kk, b[u][ch]);
                         }
                     }
-                } else {
+                    double part[kB];
+#pragma unroll
+                    for (int u = 0; u < kB; ++u) {
+                        part[u] = 0.0;
+#pragma unroll
+                        for (int ch = 0; ch < NA; ++ch)
+#pragma unroll
+                            for (int q = 0; q < V; ++q) part[u] = fma(a[ch][q], b[u][ch][q], part[u]);
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                        for (int u = 0; u < kB; ++u) part[u] += __shfl_xor_sync(0xffffffffu, part[u], o);
+#pragma unroll
+                    for (int u = 0; u < kB; ++u)
+                        if (t + u < cnt && lane == off + t + u) res = part[u];
+                }
+            } else {
+                for (int t = 0; t < cnt; ++t) {
+                    const int64_t j = SP_IDX(__shfl_sync(0xffffffffu, c_l, off + t), nb);
+                    const double* brow = Bt + j * ldt;
+                    double part = 0.0;
                     for (int64_t kk = (int64_t)lane * V; kk < K; kk += 32 * V) {
                         double b[V], aa[V];
                         ld2<V>(brow + kk, b);
@@ -117,10 +145,10 @@ k_sddmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __re
 #pragma unroll
                         for (int q = 0; q < V; ++q) part = fma(aa[q], b[q], part);
                     }
-                }
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-                if (lane == off + t) res = part;
+                    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                    if (lane == off + t) res = part;
+                }
             }
             p += cnt;
         }
