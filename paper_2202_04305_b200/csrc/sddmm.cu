@@ -40,7 +40,10 @@ k_transpose(const double* __restrict__ B, int64_t ldb, int64_t K, int64_t n, dou
 
 template <int V>
 __device__ __forceinline__ void ld2(const double* p, double* a) {
-    if (V == 2) { double2 q = *reinterpret_cast<const double2*>(p); a[0] = q.x; a[V - 1] = q.y; }
+    if (V == 4) {           // one 32-byte load (p is 32-byte aligned)
+        asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];"
+                     : "=d"(a[0]), "=d"(a[V > 1 ? 1 : 0]), "=d"(a[V > 2 ? 2 : 0]), "=d"(a[V > 3 ? 3 : 0]) : "l"(p));
+    } else if (V == 2) { double2 q = *reinterpret_cast<const double2*>(p); a[0] = q.x; a[V - 1] = q.y; }
     else a[0] = *p;
 }
 
@@ -275,6 +278,9 @@ extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const 
     if (st != SP_OK) return st;
     const bool vec2 = (K % 2 == 0) && (lda % 2 == 0) && (reinterpret_cast<uintptr_t>(A) % 16 == 0) &&
                       (reinterpret_cast<uintptr_t>(Bt) % 16 == 0);
+    // 32-byte loads when every operand row starts on a 32-byte boundary and K is a multiple of four
+    const bool vec4 = vec2 && (K % 4 == 0) && (lda % 4 == 0) && (ldt % 4 == 0) && (reinterpret_cast<uintptr_t>(A) % 32 == 0) &&
+                      (reinterpret_cast<uintptr_t>(Bt) % 32 == 0);
     const unsigned blocks = (unsigned)sp_ceil_div(part.nchunks * 32, kSThreads);
     // The kernel keeps the operand row of the outer (segment) index in registers and gathers the
     // row of the inner index: for column-major S the two operands simply trade places
@@ -291,7 +297,11 @@ extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const 
         const P* pos = static_cast<const P*>(S->pos[1]);
         const I* crd = static_cast<const I*>(S->crd[1]);
         const I* outer = dbl ? static_cast<const I*>(S->crd[0]) : nullptr;
-        if (vec2) {
+        if (vec4 && K > 64 && K <= 512) {
+            if (K <= 128) SP_SDDMM_LAUNCH(4, 1);
+            else if (K <= 256) SP_SDDMM_LAUNCH(4, 2);
+            else SP_SDDMM_LAUNCH(4, 4);
+        } else if (vec2) {
             if (K <= 64) SP_SDDMM_LAUNCH(2, 1);
             else if (K <= 128) SP_SDDMM_LAUNCH(2, 2);
             else if (K <= 256) SP_SDDMM_LAUNCH(2, 4);
