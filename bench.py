@@ -240,7 +240,7 @@ NCU_LEVELS = {
     "spmm_dcsr": {"lts_bytes": 2.402e9, "dram_bytes": 1.211e9, "source": "profiles/spmv_spmm_sddmm_full_configs.md"},
     "spmv_dcsr": {"lts_bytes": 333.8e6, "dram_bytes": 71.6e6, "source": "profiles/spmv_spmm_sddmm_full_configs.md"},
     "spmm_csr": {"lts_bytes": 0.672e9, "dram_bytes": 63.0e6, "source": "profiles/spmv_spmm_sddmm_full_configs.md"},
-    "sddmm_csr": {"lts_bytes": 3.121e9, "dram_bytes": 1.209e9, "source": "profiles/spmv_spmm_sddmm_full_configs.md"},
+    "sddmm_csr": {"lts_bytes": 3.070e9, "dram_bytes": 1.186e9, "source": "profiles/spmv_spmm_sddmm_full_configs.md"},
     "mttkrp_csf": {"lts_bytes": 3.679e9, "dram_bytes": 0.2944e9, "source": "profiles/k_mttkrp_16384cube_20M.md"},
 }
 
