@@ -176,6 +176,29 @@ __device__ __forceinline__ int64_t sp_checked_index(int64_t i, int64_t n, int li
 #define SP_IDX(i, n) (i)
 #endif
 
+// Chains of short kernels in which each needs the one before it (the packer's passes, a kernel and
+// its fix-up) are launched as programmatic dependents: the next kernel may be set up on the device
+// while its predecessor drains, and its first statement waits until that predecessor has completed
+// and its writes are visible.  Nothing triggers early: the only thing overlapped is the launch itself.
+// In a kernel launched the ordinary way the wait returns at once.
+__device__ __forceinline__ void sp_wait_for_previous_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t sp_launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ double sp_shfl(double v, int src) {
     return __shfl_sync(0xffffffffu, v, src);
 }

@@ -200,6 +200,7 @@ __device__ __forceinline__ uint32_t block256_excl_scan(uint32_t v, uint32_t* sum
 template <int BITS, bool PAY>
 __global__ void __launch_bounds__(kSortThreads)
 k_sort_upsweep(const uint64_t* __restrict__ keys, int64_t n, int shift, uint32_t* __restrict__ tilehist, int64_t ntiles) {
+    sp_wait_for_previous_kernel();
     constexpr int kSortIpt = SortShape<PAY>::kIpt, kSortTile = SortShape<PAY>::kTile;
     constexpr int RADIX = 1 << BITS;
     constexpr uint32_t mask = RADIX - 1;
@@ -252,6 +253,7 @@ constexpr int kScanChunk = 2048;
 
 __global__ void __launch_bounds__(256)
 k_sort_chunk_totals(const uint32_t* __restrict__ tilehist, int64_t ntiles, int64_t nchunks, uint32_t* __restrict__ chunk_tot) {
+    sp_wait_for_previous_kernel();
     __shared__ uint32_t sums[8];
     const uint32_t* row = tilehist + (int64_t)blockIdx.x * ntiles;
     const int64_t base = (int64_t)blockIdx.y * kScanChunk;
@@ -269,6 +271,7 @@ k_sort_chunk_totals(const uint32_t* __restrict__ tilehist, int64_t ntiles, int64
 __global__ void __launch_bounds__(256)
 k_sort_scan(uint32_t* tilehist, int64_t ntiles, int64_t nchunks, const uint32_t* __restrict__ chunk_tot,
             uint32_t* __restrict__ digit_total) {
+    sp_wait_for_previous_kernel();
     __shared__ uint32_t stage[kScanChunk];
     __shared__ uint32_t sums[8];
     uint32_t* row = tilehist + (int64_t)blockIdx.x * ntiles;
@@ -336,6 +339,7 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint64_t* __restric
                  int64_t n, int shift,
                  const uint32_t* __restrict__ tilehist, int64_t ntiles,
                  const uint32_t* __restrict__ digit_total, int split_bits) {
+    sp_wait_for_previous_kernel();
     constexpr int kSortIpt = SortShape<PAY>::kIpt, kSortTile = SortShape<PAY>::kTile;
     constexpr int RADIX = 1 << BITS;
     constexpr uint32_t mask = RADIX - 1;
@@ -463,8 +467,8 @@ sp_status sort_pass(const uint64_t* kin, const uint64_t* pin, uint64_t* kout, ui
                     uint32_t* tilehist, int64_t stiles, uint32_t* digit_total, uint32_t* chunk_tot, bool fused, int split_bits,
                     bool have_hist, cudaStream_t stream, PhaseTimer& timer) {
     if (!have_hist) {
-        if (fused) k_sort_upsweep<BITS, false><<<(unsigned)stiles, kSortThreads, 0, stream>>>(kin, n, shift, tilehist, stiles);
-        else k_sort_upsweep<BITS, true><<<(unsigned)stiles, kSortThreads, 0, stream>>>(kin, n, shift, tilehist, stiles);
+        if (fused) SP_CUDA(sp_launch_dependent(k_sort_upsweep<BITS, false>, dim3((unsigned)stiles), dim3(kSortThreads), 0, stream, kin, n, shift, tilehist, stiles));
+        else SP_CUDA(sp_launch_dependent(k_sort_upsweep<BITS, true>, dim3((unsigned)stiles), dim3(kSortThreads), 0, stream, kin, n, shift, tilehist, stiles));
         sp_count_launches(1);
     }
     timer.mark(kPhUpsweep);
@@ -472,22 +476,24 @@ sp_status sort_pass(const uint64_t* kin, const uint64_t* pin, uint64_t* kout, ui
         const int64_t nchunks = sp_ceil_div(stiles, kScanChunk);
         dim3 grid(1u << BITS, (unsigned)nchunks);
         if (nchunks > 1) {
-            k_sort_chunk_totals<<<grid, 256, 0, stream>>>(tilehist, stiles, nchunks, chunk_tot);
+            SP_CUDA(sp_launch_dependent(k_sort_chunk_totals, grid, dim3(256), 0, stream, tilehist, stiles, nchunks, chunk_tot));
             sp_count_launches(1);
         }
-        k_sort_scan<<<grid, 256, 0, stream>>>(tilehist, stiles, nchunks, chunk_tot, digit_total);
+        SP_CUDA(sp_launch_dependent(k_sort_scan, grid, dim3(256), 0, stream, tilehist, stiles, nchunks, chunk_tot, digit_total));
     }
     timer.mark(kPhScan);
     if (fused) {
         SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep<false, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)down_smem(false, BITS)));
-        k_sort_downsweep<false, BITS><<<(unsigned)stiles, kSortThreads, down_smem(false, BITS), stream>>>(
-            kin, nullptr, kout, nullptr, iout, n, shift, tilehist, stiles, digit_total, split_bits);
+        SP_CUDA(sp_launch_dependent(k_sort_downsweep<false, BITS>, dim3((unsigned)stiles), dim3(kSortThreads), down_smem(false, BITS), stream,
+                                 kin, (const uint64_t*)nullptr, kout, (uint64_t*)nullptr, iout, n, shift, (const uint32_t*)tilehist, stiles,
+                                 (const uint32_t*)digit_total, split_bits));
     } else {
         SP_CUDA(cudaFuncSetAttribute(k_sort_downsweep<true, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)down_smem(true, BITS)));
-        k_sort_downsweep<true, BITS><<<(unsigned)stiles, kSortThreads, down_smem(true, BITS), stream>>>(
-            kin, pin, kout, pout, nullptr, n, shift, tilehist, stiles, digit_total, -1);
+        SP_CUDA(sp_launch_dependent(k_sort_downsweep<true, BITS>, dim3((unsigned)stiles), dim3(kSortThreads), down_smem(true, BITS), stream,
+                                 kin, pin, kout, pout, (uint32_t*)nullptr, n, shift, (const uint32_t*)tilehist, stiles,
+                                 (const uint32_t*)digit_total, -1));
     }
     SP_LAUNCH_CHECK();
     timer.mark(kPhDownsweep);
@@ -535,6 +541,7 @@ __device__ __forceinline__ uint64_t block_excl_scan64(uint64_t v, uint64_t* sums
 template <int RANK>
 __global__ void __launch_bounds__(kCtThreads)
 k_count_flags(const uint64_t* __restrict__ keys, int64_t n, LevelPlan p, uint64_t* __restrict__ tilesum) {
+    sp_wait_for_previous_kernel();
     __shared__ uint32_t wtot[kCtThreads / 32][SP_MAX_RANK];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int64_t chunk = (int64_t)blockIdx.x * kCtTile + (int64_t)w * (32 * kCtIpt);
@@ -583,6 +590,7 @@ static_assert(kField * SP_MAX_RANK <= 64 && (1 << kField) > kCtTile, "packed per
 __global__ void __launch_bounds__(512)
 k_scan_tiles(const uint64_t* __restrict__ tilesum, int64_t ntiles, int rank, int64_t* __restrict__ tileprefix,
              int64_t* __restrict__ counts) {
+    sp_wait_for_previous_kernel();
     __shared__ uint64_t sums[16];
     const int64_t per = (ntiles + 511) / 512;
     const int64_t q0 = (int64_t)threadIdx.x * per, q1 = q0 + per < ntiles ? q0 + per : ntiles;
@@ -792,6 +800,7 @@ __global__ void __launch_bounds__(kCtThreads) k_rmin_reduce(const T* __restrict_
 
 template <typename T>
 __global__ void __launch_bounds__(512) k_rmin_tiles(T* tilemin, int64_t ntiles) {
+    sp_wait_for_previous_kernel();
     __shared__ T sums[16];
     const T ident = ~(T)0;
     T carry = ident;
@@ -807,6 +816,7 @@ __global__ void __launch_bounds__(512) k_rmin_tiles(T* tilemin, int64_t ntiles) 
 
 template <typename T>
 __global__ void __launch_bounds__(kCtThreads) k_rmin_apply(T* __restrict__ a, int64_t L, const T* __restrict__ tilecarry) {
+    sp_wait_for_previous_kernel();
     __shared__ T sums[16];
     const T ident = ~(T)0;
     int64_t r0 = (int64_t)blockIdx.x * kCtTile + (int64_t)threadIdx.x * kCtIpt;
@@ -836,8 +846,8 @@ sp_status suffix_min_inplace(void* a, int64_t L, cudaStream_t stream) {
     T* tm = ws.get<T>((size_t)ntiles);
     if (ws.failed) return SP_ERR_ALLOC;
     k_rmin_reduce<T><<<(unsigned)ntiles, kCtThreads, 0, stream>>>(static_cast<const T*>(a), L, tm);
-    k_rmin_tiles<T><<<1, 512, 0, stream>>>(tm, ntiles);
-    k_rmin_apply<T><<<(unsigned)ntiles, kCtThreads, 0, stream>>>(static_cast<T*>(a), L, tm);
+    SP_CUDA(sp_launch_dependent(k_rmin_tiles<T>, dim3(1), dim3(512), 0, stream, tm, ntiles));
+    SP_CUDA(sp_launch_dependent(k_rmin_apply<T>, dim3((unsigned)ntiles), dim3(kCtThreads), 0, stream, static_cast<T*>(a), L, (const T*)tm));
     sp_count_launches(3);
     SP_LAUNCH_CHECK();
     return SP_OK;
@@ -1021,13 +1031,13 @@ sp_status pack_impl(int rank, const int64_t* dims, int64_t nnz, const void* cons
         else vals_sorted = npasses > 0 ? reinterpret_cast<const double*>(pbuf[cur]) : coo_vals;   // no pass: one cell
 
         switch (rank) {
-            case 1: k_count_flags<1><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum); break;
-            case 2: k_count_flags<2><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum); break;
-            case 3: k_count_flags<3><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum); break;
-            case 4: k_count_flags<4><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum); break;
-            default: k_count_flags<5><<<(unsigned)ct_tiles, kCtThreads, 0, stream>>>(keys, n, plan, tilesum); break;
+            case 1: SP_CUDA(sp_launch_dependent(k_count_flags<1>, dim3((unsigned)ct_tiles), dim3(kCtThreads), 0, stream, (const uint64_t*)keys, n, plan, tilesum)); break;
+            case 2: SP_CUDA(sp_launch_dependent(k_count_flags<2>, dim3((unsigned)ct_tiles), dim3(kCtThreads), 0, stream, (const uint64_t*)keys, n, plan, tilesum)); break;
+            case 3: SP_CUDA(sp_launch_dependent(k_count_flags<3>, dim3((unsigned)ct_tiles), dim3(kCtThreads), 0, stream, (const uint64_t*)keys, n, plan, tilesum)); break;
+            case 4: SP_CUDA(sp_launch_dependent(k_count_flags<4>, dim3((unsigned)ct_tiles), dim3(kCtThreads), 0, stream, (const uint64_t*)keys, n, plan, tilesum)); break;
+            default: SP_CUDA(sp_launch_dependent(k_count_flags<5>, dim3((unsigned)ct_tiles), dim3(kCtThreads), 0, stream, (const uint64_t*)keys, n, plan, tilesum)); break;
         }
-        k_scan_tiles<<<rank, 512, 0, stream>>>(tilesum, ct_tiles, rank, tileprefix, d_counts);
+        SP_CUDA(sp_launch_dependent(k_scan_tiles, dim3(rank), dim3(512), 0, stream, (const uint64_t*)tilesum, ct_tiles, rank, tileprefix, d_counts));
         SP_LAUNCH_CHECK();
         timer.mark(kPhCount);
         sp_count_launches(3);

@@ -56,6 +56,7 @@ k_sddmm(const P* __restrict__ pos, const I* __restrict__ crd, const double* __re
         int64_t ldt, int64_t K, double* __restrict__ xv, const int64_t* __restrict__ prow,
         const int64_t* __restrict__ pnz, int64_t nchunks, int64_t na, int64_t nb) {
     // na, nb: rows of A and of Bt (used by the bounds-checking debug build only)
+    sp_wait_for_previous_kernel();      // the transpose that wrote Bt
     const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
     if (w >= nchunks) return;
     const int lane = threadIdx.x & 31;
@@ -290,9 +291,11 @@ extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const 
         const int64_t tl = lda; lda = ldt; ldt_k = tl;
     }
 #define SP_SDDMM_LAUNCH(V, NCH)                                                                                     \
-    k_sddmm<P, I, V, NCH><<<blocks, kSThreads, 0, stream>>>(pos, crd, S->val, outer, A, lda, Bt, ldt_k, K, x_vals,  \
-                                                            part.row, part.nz, part.nchunks, S->dims[S->ord[0]],   \
-                                                            S->dims[S->ord[1]])
+    sddmm_launch_st = sp_launch_dependent(k_sddmm<P, I, V, NCH>, dim3(blocks), dim3(kSThreads), 0, stream, pos, crd,  \
+                                          (const double*)S->val, outer, (const double*)A, lda, (const double*)Bt, ldt_k, K, \
+                                          x_vals, (const int64_t*)part.row, (const int64_t*)part.nz, part.nchunks,        \
+                                          S->dims[S->ord[0]], S->dims[S->ord[1]])
+    cudaError_t sddmm_launch_st = cudaSuccess;
     SP_DISPATCH_WIDTHS(S, {
         const P* pos = static_cast<const P*>(S->pos[1]);
         const I* crd = static_cast<const I*>(S->crd[1]);
@@ -311,6 +314,7 @@ extern "C" sp_status sp_sddmm(sp_tensor* S, const double* A, int64_t lda, const 
         }
     });
 #undef SP_SDDMM_LAUNCH
+    SP_CUDA(sddmm_launch_st);
     SP_LAUNCH_CHECK();
     sp_count_launches(2);
     SP_BOUNDS_RETURN(stream);

@@ -175,6 +175,7 @@ k_spmv(const P* __restrict__ pos, const I* __restrict__ crd, const double* __res
 template <typename I>
 __global__ void k_spmv_fixup(const double* __restrict__ carry_val, const int64_t* __restrict__ carry_row,
                              int64_t ntiles, const I* __restrict__ outer, double* __restrict__ y, int64_t m) {
+    sp_wait_for_previous_kernel();
     int64_t w = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (w >= ntiles) return;
     const int64_t r = carry_row[w];
@@ -501,6 +502,7 @@ template <typename I>
 __global__ void k_spmm_fixup(const double* __restrict__ carry, const int64_t* __restrict__ carry_row,
                              int64_t nchunks, const I* __restrict__ outer, int64_t N, double* __restrict__ C,
                              int64_t ldc, int64_t m) {
+    sp_wait_for_previous_kernel();
     const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
     if (w >= nchunks) return;
     const int lane = threadIdx.x & 31;
@@ -591,7 +593,8 @@ extern "C" sp_status sp_spmv(sp_tensor* A, const double* x, double* y, void* str
         if (rowmajor) {
             k_spmv<P, I, false><<<(unsigned)part.nchunks, kVThreads, 0, stream>>>(pos, crd, A->val, outer, x, y, part.row,
                                                                                   part.nz, nseg, cval, crow, m, A->dims[1]);
-            k_spmv_fixup<I><<<(unsigned)sp_ceil_div(part.nchunks, 256), 256, 0, stream>>>(cval, crow, part.nchunks, outer, y, m);
+            SP_CUDA(sp_launch_dependent(k_spmv_fixup<I>, dim3((unsigned)sp_ceil_div(part.nchunks, 256)), dim3(256), 0, stream,
+                                        (const double*)cval, (const int64_t*)crow, part.nchunks, outer, y, m));
             sp_count_launches(2);
         } else {
             k_spmv<P, I, true><<<(unsigned)part.nchunks, kVThreads, 0, stream>>>(pos, crd, A->val, outer, x, y, part.row,
@@ -700,7 +703,8 @@ extern "C" sp_status sp_spmm(sp_tensor* A, const double* B, int64_t N, int64_t l
             else
                 k_spmm_gather<P, I, 1><<<blocks, kMThreads, 0, stream>>>(pos, crd, A->val, outer, B, N, ldb, C, ldc, part.row,
                                                                          part.nz, part.nchunks, nseg, carry, crow, m, A->dims[1]);
-            k_spmm_fixup<I><<<blocks, kMThreads, 0, stream>>>(carry, crow, part.nchunks, outer, N, C, ldc, m);
+            SP_CUDA(sp_launch_dependent(k_spmm_fixup<I>, dim3(blocks), dim3(kMThreads), 0, stream, (const double*)carry,
+                                        (const int64_t*)crow, part.nchunks, outer, N, C, ldc, m));
             sp_count_launches(2);
         } else {
             (void)pos;
