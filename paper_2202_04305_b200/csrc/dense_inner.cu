@@ -17,8 +17,13 @@ constexpr int kDThreads = 256;
 constexpr int kDUnroll = 8;
 
 // One group of TPR threads per stored slice: strided dot product with kDUnroll loads in flight.
+// four blocks per SM: 64 registers, room for the sixteen 16-byte loads a thread keeps in flight
+#ifndef SP_LB_DENSE_SPMV
+#define SP_LB_DENSE_SPMV 4
+#endif
+#define SP_DENSE_SPMV_BOUNDS __launch_bounds__(kDThreads, SP_LB_DENSE_SPMV)
 template <typename I, int TPR>
-__global__ void __launch_bounds__(kDThreads)
+__global__ void SP_DENSE_SPMV_BOUNDS
 k_spmv_dense_rows(const double* __restrict__ val, const I* __restrict__ outer, int64_t nslices, int64_t inner,
                   const double* __restrict__ x, double* __restrict__ y, int64_t douter) {
     __shared__ double s_part[kDThreads / 32];
