@@ -302,7 +302,7 @@ k_sort_scan(uint32_t* tilehist, int64_t ntiles, int64_t nchunks, const uint32_t*
 
 constexpr size_t down_smem(bool pay, int bits) {
     return (size_t)(pay ? SortShape<true>::kTile : SortShape<false>::kTile) * (pay ? 16 : 8) + (size_t)kSortWarps * ((1 << bits) + 1) * 4 +
-           (size_t)((1 << bits) + 1) * 4 + (size_t)(1 << bits) * 4 + 64;
+           (size_t)(1 << bits) * 4 + 64;
 }
 
 // Ranks the warp's rounds of 32 keys: rank i = number of earlier keys of this warp with the same
@@ -347,8 +347,7 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint64_t* __restric
     uint64_t* skeys = reinterpret_cast<uint64_t*>(smem_raw);
     uint64_t* spay = skeys + kSortTile;
     uint32_t* wcnt = reinterpret_cast<uint32_t*>(PAY ? spay + kSortTile : spay);   // [warps][RADIX + 1]
-    uint32_t* dstart = wcnt + kSortWarps * (RADIX + 1);       // [RADIX + 1]
-    uint32_t* goff = dstart + (RADIX + 1);                    // [RADIX]: global position of the digit's first key minus dstart (mod 2^32)
+    uint32_t* goff = wcnt + kSortWarps * (RADIX + 1);         // [RADIX]: where the digit's keys go in the output minus where they start in the tile (mod 2^32)
     __shared__ uint32_t sums[kSortThreads / 32];
 
     const int t = threadIdx.x, w = t >> 5, lane = t & 31;
@@ -422,14 +421,16 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint64_t* __restric
     for (int q = 0; q < DPT; ++q) {
         const int d = t * DPT + q;
         if (d < RADIX) {
-            dstart[d] = ex;
+            // the warps' offsets inside the digit become positions inside the tile, so that placing a
+            // key needs one table look-up
+            for (int ww = 0; ww < kSortWarps; ++ww) wcnt[ww * (RADIX + 1) + d] += ex;
             // global base of digit d = totals of smaller digits + this tile's prefix within the digit
             goff[d] = gex + tilehist[(int64_t)d * ntiles + blockIdx.x] - ex;
             ex += tot_d[q];
             gex += gtot_d[q];
         }
     }
-    if (t == 0) dstart[RADIX] = tot_all;
+    (void)tot_all;
     __syncthreads();
 
 #pragma unroll
@@ -437,7 +438,7 @@ k_sort_downsweep(const uint64_t* __restrict__ keys_in, const uint64_t* __restric
         const int li = w * (32 * kSortIpt) + i * 32 + lane;
         const bool valid = li < tile_n;
         const uint32_t d = valid ? ((uint32_t)(key[i] >> shift) & mask) : (uint32_t)RADIX;
-        const uint32_t s = dstart[d] + mycnt[d] + ((i & 1) ? rank[i / 2] >> 16 : rank[i / 2] & 0xffffu);
+        const uint32_t s = mycnt[d] + ((i & 1) ? rank[i / 2] >> 16 : rank[i / 2] & 0xffffu);
         if (valid) {
             skeys[s] = key[i];
             if (PAY) spay[s] = pay[i];
