@@ -822,7 +822,7 @@ def main():
 
 
 # DRAM bytes (read + write) per launch from ncu captures of the current kernels (profiles/): the sort's
-# scatter pass on 20,000,000 entries read 325.9 MB and wrote 272.7 MB (algorithmic: 640 MB; the rest of the
+# scatter pass on 20,000,000 entries read 325.6 MB and wrote 273.0 MB (algorithmic: 640 MB; the rest of the
 # written lines were still in L2 when the launch ended).
 NCU_TRAFFIC = {"k_sort_downsweep": 598.6e6}
 # one radix pass over a tensor whose key and entry index do not fit 64 bits together (the 20,000,000-entry
